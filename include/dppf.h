@@ -1,0 +1,142 @@
+/*
+ * dppf.h -- C ABI of the DPPF communication-round consensus step on one GPU.
+ *
+ * The M worker replicas of a d-parameter model live in one device buffer
+ * x[M, ld] (fp32, row-major, row m = worker m).  One round
+ *   1. forms the average x_A = (1/M) sum_m x_m            (Algorithm 1, last line),
+ *   2. measures r_m = ||x_m - x_A||_2 for every worker     (norm in the single-line
+ *      update, Sec. 5; the consensus distance logged in the ablations),
+ *   3. applies x_m <- x_m + (x_A - x_m)(alpha - lambda / r_m) to every replica,
+ *      all workers using the same pre-round x_A            (single-line pull-push
+ *      update, Sec. 5; first display of the proof of Theorem 1).
+ * x_A is never stored: it is recomputed per tile in registers.
+ *
+ * Conventions for every entry point
+ *   - Pointers named x, v, g, norms_out, ws, x_dev are DEVICE pointers owned by the
+ *     caller; *_host pointers are HOST pointers.  The library allocates nothing.
+ *   - Layout: row stride ld >= d with ld % 32 == 0, base pointers 128-byte
+ *     aligned, so every row starts on a 128-byte boundary.  Columns d..ld-1 are
+ *     never read into a result and never written.
+ *   - Updates are in place and asynchronous on `cuda_stream` (a cudaStream_t cast
+ *     to void*; NULL = the legacy default stream).  Calls that touch the same
+ *     buffers or the same workspace must be ordered on one stream.
+ *   - x, v and g must not overlap.
+ *   - Scalars are fp32 and must be finite; alpha outside (0,1] and negative
+ *     lambda are accepted (the invariants alpha = 0 and lambda = 0 need them).
+ *   - Return value: a dppf_status.  On any value other than DPPF_OK nothing has
+ *     been launched and no buffer has been touched.
+ *   - Zero distance (r_m == 0, e.g. M == 1 or identical replicas): the paper
+ *     leaves 0/0 undefined; here no push is applied, the replica is left
+ *     bit-for-bit unchanged and r_m = 0 is reported.
+ *   - Results are run-to-run reproducible on a given GPU model: the tile-to-block
+ *     map is static and every reduction runs in a fixed order (no float atomics).
+ */
+#ifndef DPPF_H
+#define DPPF_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DPPF_OK = 0,
+    DPPF_ERR_INVALID_ARG = 1,  /* null pointer, M/d/ld out of range, non-finite scalar, overlap */
+    DPPF_ERR_ALIGNMENT = 2,    /* base pointer not 128-byte aligned or ld % 32 != 0 */
+    DPPF_ERR_WORKSPACE = 3,    /* ws_bytes < dppf_workspace_bytes(M, d) */
+    DPPF_ERR_CUDA = 4,         /* a CUDA runtime call or launch failed */
+    DPPF_ERR_TIMEOUT = 5       /* reserved: a bounded device-side wait gave up */
+} dppf_status;
+
+/* Largest worker count handled (rows of x). */
+#define DPPF_MAX_WORKERS 1024
+
+/* Kernel schedule selector for the *_ex entry points. */
+#define DPPF_PATH_AUTO 0        /* library picks */
+#define DPPF_PATH_TWO_KERNEL 1  /* distance pass, then update pass, as two launches */
+#define DPPF_PATH_COOPERATIVE 2 /* one persistent cooperative launch with a grid-wide barrier */
+
+/*
+ * Scratch size in bytes for a round on M replicas of length d (the per-block
+ * partial sums of squared distances of step 2, plus a small header).  Returns 0
+ * for invalid M or d.  The workspace needs no initialisation and may be reused
+ * by later calls on the same stream.
+ */
+size_t dppf_workspace_bytes(int M, int64_t d);
+
+/*
+ * One pull-push round in place on x[M, ld] (steps 1-3 above; Sec. 5 single-line
+ * update with x_C = x_A).  norms_out: NULL, or device fp32[M] that receives the
+ * PRE-update distances r_m (the consensus distance the paper logs per worker).
+ */
+int dppf_consensus(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
+                   float *norms_out, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Same, with an explicit kernel schedule (DPPF_PATH_*).  Both schedules give
+ * bit-identical results. */
+int dppf_consensus_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
+                      float *norms_out, void *ws, size_t ws_bytes, int path, void *cuda_stream);
+
+/*
+ * One local optimiser step between rounds, in place, for all M workers
+ * (Algorithm 1, the local update line; the experiments run SGD with momentum
+ * and weight decay, whose recurrence the paper does not print -- the coupled
+ * form is used):   g~ = g + weight_decay * x ;  v <- momentum * v + g~ ;
+ *                  x <- x - lr * v.
+ * v[M, ld] is the momentum buffer (0 before the first step), g[M, ld] the
+ * gradients (read only).  Same layout rules as x.
+ */
+int dppf_local_step(float *x, float *v, const float *g, int M, int64_t d, int64_t ld,
+                    float lr, float momentum, float weight_decay, void *cuda_stream);
+
+/*
+ * The last local step before a round fused with the round: exactly
+ * dppf_local_step followed by dppf_consensus, but the distance pass reads x, v, g
+ * once and produces the stepped replicas and their distances together.
+ */
+int dppf_local_step_and_consensus(float *x, float *v, const float *g, int M, int64_t d,
+                                  int64_t ld, float lr, float momentum, float weight_decay,
+                                  float alpha, float lambda, float *norms_out, void *ws,
+                                  size_t ws_bytes, void *cuda_stream);
+
+int dppf_local_step_and_consensus_ex(float *x, float *v, const float *g, int M, int64_t d,
+                                     int64_t ld, float lr, float momentum, float weight_decay,
+                                     float alpha, float lambda, float *norms_out, void *ws,
+                                     size_t ws_bytes, int path, void *cuda_stream);
+
+/*
+ * Round on replicas that live in HOST memory (the arrangement the paper's
+ * limitations section mentions: parameters kept off the accelerator).  Copies
+ * x_host[M, ld] into the caller's device staging buffer x_dev[M, ld], runs
+ * dppf_consensus there, copies the updated replicas back into x_host and, if
+ * norms_host != NULL, the M pre-update distances into norms_host (host fp32[M]).
+ * All copies are cudaMemcpyAsync on `cuda_stream`; pinned host memory makes them
+ * truly asynchronous.  The results are valid once the stream has been
+ * synchronised.  x_host needs no particular alignment; x_dev follows the device
+ * layout rules.  norms staging uses the workspace.
+ */
+int dppf_consensus_host(float *x_host, int M, int64_t d, int64_t ld, float alpha, float lambda,
+                        float *norms_host, float *x_dev, void *ws, size_t ws_bytes,
+                        void *cuda_stream);
+
+/*
+ * Synchronises `cuda_stream` and returns the status word the kernels keep in the
+ * workspace header: DPPF_OK, or DPPF_ERR_WORKSPACE if the update pass found a
+ * header that its distance pass did not write (workspace overwritten between the
+ * two), in which case x was left unchanged.  DPPF_ERR_CUDA if the stream failed.
+ */
+int dppf_device_status(const void *ws, void *cuda_stream);
+
+/* Static, human-readable name of a dppf_status. */
+const char *dppf_status_string(int status);
+
+/* Number of kernel launches the given call shape issues (for launch accounting):
+ * fused != 0 selects dppf_local_step_and_consensus. */
+int dppf_launch_count(int M, int64_t d, int path, int fused);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DPPF_H */

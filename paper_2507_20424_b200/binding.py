@@ -1,0 +1,161 @@
+"""ctypes binding of ``libdppf.so``: argument marshalling only.
+
+Every function takes torch CUDA tensors (used purely as device memory) and
+passes raw pointers, sizes and the current CUDA stream to the C entry point of
+the same name (``include/dppf.h``).  There is no CPU fallback: if the library
+is missing or a call returns an error status, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+PATH_AUTO, PATH_TWO_KERNEL, PATH_COOPERATIVE = 0, 1, 2
+OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+
+EXPORTS = ("dppf_workspace_bytes", "dppf_consensus", "dppf_consensus_ex", "dppf_local_step",
+           "dppf_local_step_and_consensus", "dppf_local_step_and_consensus_ex",
+           "dppf_consensus_host", "dppf_device_status", "dppf_status_string", "dppf_launch_count")
+
+_lib = None
+
+
+class DppfError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+def library_path() -> str:
+    return _build.LIB_PATH
+
+
+def load(rebuild_if_stale: bool = False) -> ctypes.CDLL:
+    """Load the shared library (building it first only when asked to)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if rebuild_if_stale:
+        _build.build()
+    if not os.path.exists(_build.LIB_PATH):
+        raise RuntimeError(f"{_build.LIB_PATH} not found: build it with "
+                           "`python -m paper_2507_20424_b200.build` (no CPU fallback exists)")
+    lib = ctypes.CDLL(_build.LIB_PATH)
+    vp, f32, i32, i64, sz = ctypes.c_void_p, ctypes.c_float, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t
+    lib.dppf_workspace_bytes.argtypes = [i32, i64]
+    lib.dppf_workspace_bytes.restype = sz
+    lib.dppf_consensus.argtypes = [vp, i32, i64, i64, f32, f32, vp, vp, sz, vp]
+    lib.dppf_consensus_ex.argtypes = [vp, i32, i64, i64, f32, f32, vp, vp, sz, i32, vp]
+    lib.dppf_local_step.argtypes = [vp, vp, vp, i32, i64, i64, f32, f32, f32, vp]
+    lib.dppf_local_step_and_consensus.argtypes = [vp, vp, vp, i32, i64, i64, f32, f32, f32, f32, f32, vp, vp, sz, vp]
+    lib.dppf_local_step_and_consensus_ex.argtypes = [vp, vp, vp, i32, i64, i64, f32, f32, f32, f32, f32, vp, vp, sz, i32, vp]
+    lib.dppf_consensus_host.argtypes = [vp, i32, i64, i64, f32, f32, vp, vp, vp, sz, vp]
+    lib.dppf_device_status.argtypes = [vp, vp]
+    lib.dppf_status_string.argtypes = [i32]
+    lib.dppf_status_string.restype = ctypes.c_char_p
+    lib.dppf_launch_count.argtypes = [i32, i64, i32, i32]
+    for name in ("dppf_consensus", "dppf_consensus_ex", "dppf_local_step", "dppf_local_step_and_consensus",
+                 "dppf_local_step_and_consensus_ex", "dppf_consensus_host", "dppf_device_status",
+                 "dppf_launch_count"):
+        getattr(lib, name).restype = i32
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load().dppf_status_string(int(status)).decode()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != OK:
+        raise DppfError(rc, where)
+
+
+def _dims(x: torch.Tensor, d):
+    if x.dim() != 2 or x.dtype != torch.float32 or not x.is_cuda or x.stride(1) != 1:
+        raise ValueError("expected a 2-D fp32 CUDA tensor with unit column stride")
+    M, ld = x.shape[0], x.stride(0)
+    return M, (x.shape[1] if d is None else int(d)), ld
+
+
+def workspace_bytes(M: int, d: int) -> int:
+    return int(load().dppf_workspace_bytes(int(M), int(d)))
+
+
+def alloc_workspace(M: int, d: int, device="cuda") -> torch.Tensor:
+    n = workspace_bytes(M, d)
+    if n == 0:
+        raise ValueError("invalid M or d")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def alloc_rows(M: int, d: int, device="cuda", fill=None) -> torch.Tensor:
+    """[M, ld] fp32 device buffer with 128-byte rows (ld = d rounded up to 32)."""
+    ld = (int(d) + 31) // 32 * 32
+    t = torch.empty((M, ld), dtype=torch.float32, device=device)
+    if fill is not None:
+        t.fill_(fill)
+    return t
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def dppf_consensus(x, alpha, lam, norms_out=None, ws=None, d=None, path=PATH_AUTO):
+    """One pull-push round in place on ``x[M, ld]``; returns the workspace used."""
+    M, d, ld = _dims(x, d)
+    ws = alloc_workspace(M, d, x.device) if ws is None else ws
+    rc = load().dppf_consensus_ex(x.data_ptr(), M, d, ld, alpha, lam, _ptr(norms_out),
+                                  ws.data_ptr(), ws.numel(), int(path), _stream())
+    _check(rc, "dppf_consensus")
+    return ws
+
+
+def dppf_local_step(x, v, g, lr, momentum, weight_decay, d=None):
+    M, d, ld = _dims(x, d)
+    for t in (v, g):
+        if _dims(t, d) != (M, d, ld):
+            raise ValueError("x, v and g must share shape and row stride")
+    _check(load().dppf_local_step(x.data_ptr(), v.data_ptr(), g.data_ptr(), M, d, ld,
+                                  lr, momentum, weight_decay, _stream()), "dppf_local_step")
+
+
+def dppf_local_step_and_consensus(x, v, g, lr, momentum, weight_decay, alpha, lam,
+                                  norms_out=None, ws=None, d=None, path=PATH_AUTO):
+    M, d, ld = _dims(x, d)
+    for t in (v, g):
+        if _dims(t, d) != (M, d, ld):
+            raise ValueError("x, v and g must share shape and row stride")
+    ws = alloc_workspace(M, d, x.device) if ws is None else ws
+    rc = load().dppf_local_step_and_consensus_ex(
+        x.data_ptr(), v.data_ptr(), g.data_ptr(), M, d, ld, lr, momentum, weight_decay,
+        alpha, lam, _ptr(norms_out), ws.data_ptr(), ws.numel(), int(path), _stream())
+    _check(rc, "dppf_local_step_and_consensus")
+    return ws
+
+
+def dppf_consensus_host(x_host, alpha, lam, norms_host, x_dev, ws, d=None):
+    """Round on host-resident replicas (pinned CPU tensors), staged through ``x_dev``."""
+    M, d, ld = _dims(x_dev, d)
+    if x_host.dtype != torch.float32 or x_host.is_cuda or x_host.shape[0] != M or x_host.stride(0) != ld:
+        raise ValueError("x_host must be a CPU fp32 tensor with the row stride of x_dev")
+    rc = load().dppf_consensus_host(x_host.data_ptr(), M, d, ld, alpha, lam, _ptr(norms_host),
+                                    x_dev.data_ptr(), ws.data_ptr(), ws.numel(), _stream())
+    _check(rc, "dppf_consensus_host")
+
+
+def dppf_device_status(ws) -> int:
+    return int(load().dppf_device_status(ws.data_ptr(), _stream()))
+
+
+def launch_count(M: int, d: int, path=PATH_AUTO, fused=False) -> int:
+    return int(load().dppf_launch_count(int(M), int(d), int(path), int(bool(fused))))

@@ -1,0 +1,809 @@
+// DPPF consensus round for one B200 (sm_100a): kernels and the C ABI of include/dppf.h.
+//
+// Data layout: x[M, ld] fp32, one row per worker, rows 128-byte aligned.  A "vector" is
+// one float4 (four consecutive columns of one row); a thread always handles the same
+// vector index in all M rows, so the average over workers (Algorithm 1, last line) is a
+// purely per-thread quantity and is never written to memory.
+//
+// Round = distance pass + update pass (single-line pull-push update, Sec. 5):
+//   distance pass  reads the M rows once, forms the deviations dev_m = x_m - x_A per
+//                  column and accumulates sum(dev_m^2) per worker; each block leaves M
+//                  fp64 partial sums in the workspace.
+//   update pass    every block first adds the per-block partials in block order (the
+//                  same order everywhere, so the result is identical in all blocks and
+//                  from run to run), takes r_m = sqrt(.), c_m = alpha - lambda / r_m,
+//                  then re-reads the rows, recomputes dev_m with the same instructions
+//                  and writes x_m - c_m * dev_m  ( = x_m + (x_A - x_m) c_m ).
+// The update pass walks the tiles in reverse so that it starts on the lines the
+// distance pass touched last (still in L2) and ends where the next round begins.
+//
+// Deviations use a shifted mean: e_m = x_m - x_0, ebar = (sum_m e_m)/M, dev_0 = -ebar,
+// dev_m = e_m - ebar.  Identical replicas give dev_m == 0 exactly for every M, which
+// makes the zero-distance round leave x bit-for-bit unchanged.
+#include "dppf.h"
+
+#include <cooperative_groups.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstdint>
+
+namespace cg = cooperative_groups;
+
+namespace {
+
+constexpr int kThreads = 256;            // threads per block, all kernels
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxTemplateM = 16;        // worker counts with register-resident kernels
+constexpr int kMaxBlocksSmallM = 2048;   // partial-sum slots reserved per worker, M <= 16
+constexpr int kMaxBlocksLargeM = 512;    // ... and for the generic kernels
+constexpr size_t kHeaderBytes = 256;
+constexpr unsigned kMagic = 0x44505046u; // "DPPF"
+
+struct WsHeader {
+    int status;       // dppf_status seen by the kernels
+    unsigned magic;   // written by the distance pass, checked by the update pass
+    int grid;         // blocks that wrote partials
+    int M;
+};
+
+struct RoundArgs {
+    float *x;
+    float *v;         // fused local step only
+    const float *g;   // fused local step only
+    long long d, ld, nvec;   // nvec = d / 4 full float4 groups per row
+    float alpha, lambda, lr, mu, wd;
+    float *norms_out; // may be null
+    float *norms_stage; // fp32[M] inside the workspace (always written)
+    WsHeader *hdr;
+    double *partials; // [grid, M]
+    int M;            // runtime copy (generic kernels)
+};
+
+// ---------------------------------------------------------------- memory access helpers
+
+__device__ __forceinline__ float4 ld_keep(const float *p) {   // normal L2 priority, skip L1
+    return __ldcg(reinterpret_cast<const float4 *>(p));
+}
+__device__ __forceinline__ float4 ld_last_use(const float *p) {  // evict-first: dead after this read
+    return __ldcs(reinterpret_cast<const float4 *>(p));
+}
+__device__ __forceinline__ void st_keep(float *p, float4 v) {
+    __stcg(reinterpret_cast<float4 *>(p), v);
+}
+
+// ---------------------------------------------------------------- arithmetic helpers
+// Explicitly rounded operations: the compiler may not re-associate or contract them, so
+// the distance pass and the update pass see bit-identical deviations.
+
+__device__ __forceinline__ float4 sub4(float4 a, float4 b) {
+    return make_float4(__fsub_rn(a.x, b.x), __fsub_rn(a.y, b.y), __fsub_rn(a.z, b.z), __fsub_rn(a.w, b.w));
+}
+__device__ __forceinline__ float4 add4(float4 a, float4 b) {
+    return make_float4(__fadd_rn(a.x, b.x), __fadd_rn(a.y, b.y), __fadd_rn(a.z, b.z), __fadd_rn(a.w, b.w));
+}
+__device__ __forceinline__ float4 scale4(float4 a, float s) {
+    return make_float4(__fmul_rn(a.x, s), __fmul_rn(a.y, s), __fmul_rn(a.z, s), __fmul_rn(a.w, s));
+}
+__device__ __forceinline__ float sq_acc(float acc, float4 d) {
+    acc = __fmaf_rn(d.x, d.x, acc);
+    acc = __fmaf_rn(d.y, d.y, acc);
+    acc = __fmaf_rn(d.z, d.z, acc);
+    acc = __fmaf_rn(d.w, d.w, acc);
+    return acc;
+}
+// x - c * dev
+__device__ __forceinline__ float4 apply4(float4 x, float4 dev, float c) {
+    return make_float4(__fmaf_rn(-c, dev.x, x.x), __fmaf_rn(-c, dev.y, x.y),
+                       __fmaf_rn(-c, dev.z, x.z), __fmaf_rn(-c, dev.w, x.w));
+}
+// Local optimiser step on one element: g~ = g + wd x ; v' = mu v + g~ ; x' = x - lr v'.
+__device__ __forceinline__ void sgd1(float &x, float &v, float g, float lr, float mu, float wd) {
+    float gt = __fmaf_rn(wd, x, g);
+    v = __fmaf_rn(mu, v, gt);
+    x = __fmaf_rn(-lr, v, x);
+}
+__device__ __forceinline__ void sgd4(float4 &x, float4 &v, float4 g, float lr, float mu, float wd) {
+    sgd1(x.x, v.x, g.x, lr, mu, wd);
+    sgd1(x.y, v.y, g.y, lr, mu, wd);
+    sgd1(x.z, v.z, g.z, lr, mu, wd);
+    sgd1(x.w, v.w, g.w, lr, mu, wd);
+}
+
+// Shifted mean of one vector over the M rows: ebar = (sum_{m>=1} (x_m - x_0)) / M, so that
+// x_A = x_0 + ebar and the deviation of row m is dev_m = (x_m - x_0) - ebar (dev_0 = -ebar).
+template <int M>
+__device__ __forceinline__ float4 shifted_mean(const float4 (&xv)[M]) {
+    const float inv_m = 1.0f / (float)M;
+    float4 esum = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int m = 1; m < M; ++m) esum = add4(esum, sub4(xv[m], xv[0]));
+    return scale4(esum, inv_m);
+}
+__device__ __forceinline__ float4 deviation(float4 xm, float4 x0, float4 ebar, int m) {
+    if (m == 0) return make_float4(-ebar.x, -ebar.y, -ebar.z, -ebar.w);
+    return sub4(sub4(xm, x0), ebar);
+}
+
+__device__ __forceinline__ double warp_sum(double a) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    return a;   // butterfly: every lane holds the same bits
+}
+
+// Coefficient of the single-line update; zero distance -> no push (replica unchanged).
+__device__ __forceinline__ float coefficient(double S, float alpha, float lambda, float *r_out) {
+    double r = sqrt(S);
+    *r_out = (float)r;
+    double c = (r > 0.0) ? (double)alpha - (double)lambda / r : (double)alpha;
+    return (float)c;
+}
+
+// ---------------------------------------------------------------- register-resident kernels (M <= 16)
+
+template <int M>
+struct Tuning {
+    // vectors per thread and tile iteration: keeps >= 64 bytes per row group in flight per thread
+    static constexpr int kUnroll = (M <= 2) ? 4 : (M <= 4) ? 2 : 1;
+    // blocks per SM the compiler must allow (register cap 64 / 85 / 128 per thread)
+    static constexpr int kMinBlocks = (M <= 4) ? 4 : (M <= 8) ? 3 : 2;
+};
+
+// Scalar tail: columns 4*nvec .. d-1 (at most three), handled by one thread of block 0.
+template <int M, bool kLocalStep>
+__device__ __forceinline__ void tail_distance(const RoundArgs &a, float (&acc)[M]) {
+    const float inv_m = 1.0f / (float)M;
+    for (long long i = a.nvec * 4; i < a.d; ++i) {
+        float xs[M];
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            float xi = a.x[m * a.ld + i];
+            if (kLocalStep) {
+                float vi = a.v[m * a.ld + i];
+                sgd1(xi, vi, a.g[m * a.ld + i], a.lr, a.mu, a.wd);
+                a.v[m * a.ld + i] = vi;
+                a.x[m * a.ld + i] = xi;
+            }
+            xs[m] = xi;
+        }
+        float esum = 0.f;
+#pragma unroll
+        for (int m = 1; m < M; ++m) { xs[m] = __fsub_rn(xs[m], xs[0]); esum = __fadd_rn(esum, xs[m]); }
+        const float ebar = __fmul_rn(esum, inv_m);
+        acc[0] = __fmaf_rn(ebar, ebar, acc[0]);
+#pragma unroll
+        for (int m = 1; m < M; ++m) { float dv = __fsub_rn(xs[m], ebar); acc[m] = __fmaf_rn(dv, dv, acc[m]); }
+    }
+}
+
+template <int M>
+__device__ __forceinline__ void tail_update(const RoundArgs &a, const float *c) {
+    const float inv_m = 1.0f / (float)M;
+    for (long long i = a.nvec * 4; i < a.d; ++i) {
+        float xs[M], dv[M];
+#pragma unroll
+        for (int m = 0; m < M; ++m) xs[m] = a.x[m * a.ld + i];
+        float esum = 0.f;
+#pragma unroll
+        for (int m = 1; m < M; ++m) { dv[m] = __fsub_rn(xs[m], xs[0]); esum = __fadd_rn(esum, dv[m]); }
+        const float ebar = __fmul_rn(esum, inv_m);
+        dv[0] = -ebar;
+#pragma unroll
+        for (int m = 1; m < M; ++m) dv[m] = __fsub_rn(dv[m], ebar);
+#pragma unroll
+        for (int m = 0; m < M; ++m) a.x[m * a.ld + i] = __fmaf_rn(-c[m], dv[m], xs[m]);
+    }
+}
+
+// Distance pass body.  Tile t of the block = vectors [(t*U+u)*kThreads + tid], u < U.
+template <int M, bool kLocalStep>
+__device__ __forceinline__ void distance_pass(const RoundArgs &a, double *s_red /* [kWarps][M] */) {
+    constexpr int U = Tuning<M>::kUnroll;
+    const long long tile_vecs = (long long)kThreads * U;
+    const long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
+    float acc[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) acc[m] = 0.f;
+
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        float4 xv[U][M];
+        bool live[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long long j = (t * U + u) * kThreads + threadIdx.x;
+            live[u] = j < a.nvec;
+            if (live[u]) {
+#pragma unroll
+                for (int m = 0; m < M; ++m) {
+                    const long long off = m * a.ld + j * 4;
+                    if (kLocalStep) {
+                        float4 xr = ld_last_use(a.x + off);
+                        float4 vr = ld_last_use(a.v + off);
+                        float4 gr = ld_last_use(a.g + off);
+                        sgd4(xr, vr, gr, a.lr, a.mu, a.wd);
+                        st_keep(a.v + off, vr);
+                        st_keep(a.x + off, xr);
+                        xv[u][m] = xr;
+                    } else {
+                        xv[u][m] = ld_keep(a.x + off);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (live[u]) {
+                const float4 ebar = shifted_mean<M>(xv[u]);
+#pragma unroll
+                for (int m = 0; m < M; ++m) acc[m] = sq_acc(acc[m], deviation(xv[u][m], xv[u][0], ebar, m));
+            }
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) tail_distance<M, kLocalStep>(a, acc);
+
+    // thread -> warp (butterfly, fp64) -> block (warp order) -> one fp64 partial per worker
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+        double s = warp_sum((double)acc[m]);
+        if (lane == 0) s_red[warp * M + m] = s;
+    }
+    __syncthreads();
+    if (threadIdx.x < M) {
+        double s = 0.0;
+        for (int w = 0; w < kWarps; ++w) s += s_red[w * M + threadIdx.x];
+        a.partials[(long long)blockIdx.x * M + threadIdx.x] = s;
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        a.hdr->status = DPPF_OK;
+        a.hdr->magic = kMagic;
+        a.hdr->grid = (int)gridDim.x;
+        a.hdr->M = M;
+    }
+}
+
+// Cross-block sum in block order, identical in every block; fills s_c[M] and reports r_m.
+// Returns false if the workspace header does not describe this launch.
+__device__ __forceinline__ bool finalise(const RoundArgs &a, int M, int nblocks, float *s_c, int *s_ok) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0)
+        *s_ok = (a.hdr->magic == kMagic && a.hdr->grid == nblocks && a.hdr->M == M) ? 1 : 0;
+    for (int m = warp; m < M; m += kWarps) {
+        double s = 0.0;
+        for (int b = lane; b < nblocks; b += 32) s += __ldcg(a.partials + (long long)b * M + m);
+        s = warp_sum(s);
+        if (lane == 0) {
+            float r;
+            s_c[m] = coefficient(s, a.alpha, a.lambda, &r);
+            if (blockIdx.x == 0) {
+                a.norms_stage[m] = r;
+                if (a.norms_out) a.norms_out[m] = r;
+            }
+        }
+    }
+    __syncthreads();
+    if (!*s_ok && blockIdx.x == 0 && threadIdx.x == 0) a.hdr->status = DPPF_ERR_WORKSPACE;
+    return *s_ok != 0;
+}
+
+template <int M>
+__device__ __forceinline__ void update_pass(const RoundArgs &a, const float *s_c) {
+    constexpr int U = Tuning<M>::kUnroll;
+    const long long tile_vecs = (long long)kThreads * U;
+    const long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
+    const float *c = s_c;
+    if (ntiles > blockIdx.x) {
+        // last tile of this block's static sequence, then backwards
+        long long t = blockIdx.x + (ntiles - 1 - blockIdx.x) / gridDim.x * gridDim.x;
+        for (; t >= 0; t -= gridDim.x) {
+            float4 xv[U][M];
+            bool live[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const long long j = (t * U + u) * kThreads + threadIdx.x;
+                live[u] = j < a.nvec;
+                if (live[u]) {
+#pragma unroll
+                    for (int m = 0; m < M; ++m) xv[u][m] = ld_last_use(a.x + m * a.ld + j * 4);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (live[u]) {
+                    const long long j = (t * U + u) * kThreads + threadIdx.x;
+                    const float4 ebar = shifted_mean<M>(xv[u]);
+#pragma unroll
+                    for (int m = 0; m < M; ++m)
+                        st_keep(a.x + m * a.ld + j * 4,
+                                apply4(xv[u][m], deviation(xv[u][m], xv[u][0], ebar, m), c[m]));
+                }
+            }
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) tail_update<M>(a, c);
+}
+
+template <int M, bool kLocalStep>
+__global__ void __launch_bounds__(kThreads, Tuning<M>::kMinBlocks) distance_kernel(const RoundArgs a) {
+    __shared__ double s_red[kWarps * M];
+    distance_pass<M, kLocalStep>(a, s_red);
+}
+
+template <int M>
+__global__ void __launch_bounds__(kThreads, Tuning<M>::kMinBlocks) update_kernel(const RoundArgs a, int nblocks_a) {
+    __shared__ float s_c[M];
+    __shared__ int s_ok;
+    if (!finalise(a, M, nblocks_a, s_c, &s_ok)) return;
+    update_pass<M>(a, s_c);
+}
+
+// One persistent launch: distance pass, grid-wide barrier, update pass.  Launched with
+// cudaLaunchCooperativeKernel, which refuses the launch unless all blocks are co-resident.
+template <int M, bool kLocalStep>
+__global__ void __launch_bounds__(kThreads, Tuning<M>::kMinBlocks) round_kernel(const RoundArgs a) {
+    __shared__ double s_red[kWarps * M];
+    __shared__ float s_c[M];
+    __shared__ int s_ok;
+    distance_pass<M, kLocalStep>(a, s_red);
+    cg::this_grid().sync();
+    if (!finalise(a, M, (int)gridDim.x, s_c, &s_ok)) return;
+    update_pass<M>(a, s_c);
+}
+
+// ---------------------------------------------------------------- generic kernels (16 < M <= 1024)
+// Rows are streamed twice per vector (second time from L1/L2); per-worker sums live in
+// shared memory, one fp32 slot per (warp, worker), so no thread needs M registers.
+
+template <bool kLocalStep>
+__global__ void __launch_bounds__(kThreads) distance_kernel_generic(const RoundArgs a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *s_acc = reinterpret_cast<float *>(smem_raw);               // [kWarps][M]
+    const int M = a.M, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float inv_m = 1.0f / (float)M;
+    for (int i = threadIdx.x; i < kWarps * M; i += kThreads) s_acc[i] = 0.f;
+    __syncthreads();
+    float *my_acc = s_acc + warp * M;
+    const long long ntiles = (a.nvec + kThreads - 1) / kThreads;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        const long long j = t * kThreads + threadIdx.x;
+        const bool live = j < a.nvec;
+        float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), esum = x0;
+        if (live) {
+            for (int m = 0; m < M; ++m) {
+                const long long off = m * a.ld + j * 4;
+                float4 xr = *reinterpret_cast<const float4 *>(a.x + off);
+                if (kLocalStep) {
+                    float4 vr = ld_last_use(a.v + off), gr = ld_last_use(a.g + off);
+                    sgd4(xr, vr, gr, a.lr, a.mu, a.wd);
+                    st_keep(a.v + off, vr);
+                    *reinterpret_cast<float4 *>(a.x + off) = xr;
+                }
+                if (m == 0) x0 = xr; else esum = add4(esum, sub4(xr, x0));
+            }
+        }
+        const float4 ebar = scale4(esum, inv_m);
+        for (int m = 0; m < M; ++m) {
+            float q = 0.f;
+            if (live) {
+                float4 dv;
+                if (m == 0) dv = make_float4(-ebar.x, -ebar.y, -ebar.z, -ebar.w);
+                else dv = sub4(sub4(*reinterpret_cast<const float4 *>(a.x + m * a.ld + j * 4), x0), ebar);
+                q = sq_acc(0.f, dv);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+            if (lane == 0) my_acc[m] += q;
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {      // scalar tail columns
+        for (long long i = a.nvec * 4; i < a.d; ++i) {
+            float x0s = 0.f, esum = 0.f;
+            for (int m = 0; m < M; ++m) {
+                float xi = a.x[m * a.ld + i];
+                if (kLocalStep) {
+                    float vi = a.v[m * a.ld + i];
+                    sgd1(xi, vi, a.g[m * a.ld + i], a.lr, a.mu, a.wd);
+                    a.v[m * a.ld + i] = vi;
+                    a.x[m * a.ld + i] = xi;
+                }
+                if (m == 0) x0s = xi; else esum = __fadd_rn(esum, __fsub_rn(xi, x0s));
+            }
+            const float ebar = __fmul_rn(esum, inv_m);
+            for (int m = 0; m < M; ++m) {
+                float dv = (m == 0) ? -ebar : __fsub_rn(__fsub_rn(a.x[m * a.ld + i], x0s), ebar);
+                my_acc[m] = __fmaf_rn(dv, dv, my_acc[m]);
+            }
+        }
+    }
+    __syncthreads();
+    for (int m = threadIdx.x; m < M; m += kThreads) {
+        double s = 0.0;
+        for (int w = 0; w < kWarps; ++w) s += (double)s_acc[w * M + m];
+        a.partials[(long long)blockIdx.x * M + m] = s;
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        a.hdr->status = DPPF_OK;
+        a.hdr->magic = kMagic;
+        a.hdr->grid = (int)gridDim.x;
+        a.hdr->M = M;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) update_kernel_generic(const RoundArgs a, int nblocks_a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *s_c = reinterpret_cast<float *>(smem_raw);                 // [M]
+    __shared__ int s_ok;
+    const int M = a.M;
+    const float inv_m = 1.0f / (float)M;
+    if (!finalise(a, M, nblocks_a, s_c, &s_ok)) return;
+    const long long ntiles = (a.nvec + kThreads - 1) / kThreads;
+    if (ntiles > blockIdx.x) {
+        long long t = blockIdx.x + (ntiles - 1 - blockIdx.x) / gridDim.x * gridDim.x;
+        for (; t >= 0; t -= gridDim.x) {
+            const long long j = t * kThreads + threadIdx.x;
+            if (j >= a.nvec) continue;
+            float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), esum = x0;
+            for (int m = 0; m < M; ++m) {
+                float4 xr = *reinterpret_cast<const float4 *>(a.x + m * a.ld + j * 4);
+                if (m == 0) x0 = xr; else esum = add4(esum, sub4(xr, x0));
+            }
+            const float4 ebar = scale4(esum, inv_m);
+            for (int m = M - 1; m >= 0; --m) {       // row 0 last: the others still need x0 (in a register)
+                float *p = a.x + m * a.ld + j * 4;
+                float4 xr = (m == 0) ? x0 : *reinterpret_cast<const float4 *>(p);
+                float4 dv = (m == 0) ? make_float4(-ebar.x, -ebar.y, -ebar.z, -ebar.w) : sub4(sub4(xr, x0), ebar);
+                st_keep(p, apply4(xr, dv, s_c[m]));
+            }
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (long long i = a.nvec * 4; i < a.d; ++i) {
+            float x0s = a.x[i], esum = 0.f;
+            for (int m = 1; m < M; ++m) esum = __fadd_rn(esum, __fsub_rn(a.x[m * a.ld + i], x0s));
+            const float ebar = __fmul_rn(esum, inv_m);
+            for (int m = M - 1; m >= 0; --m) {
+                float xi = a.x[m * a.ld + i];
+                float dv = (m == 0) ? -ebar : __fsub_rn(__fsub_rn(xi, x0s), ebar);
+                a.x[m * a.ld + i] = __fmaf_rn(-s_c[m], dv, xi);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------- stand-alone local step
+
+__global__ void __launch_bounds__(kThreads) local_step_kernel(float *x, float *v, const float *g, long long d,
+                                                              long long ld, long long nvec, float lr, float mu,
+                                                              float wd) {
+    const long long row = (long long)blockIdx.y * ld;
+    float *xr = x + row, *vr = v + row;
+    const float *gr = g + row;
+    for (long long j = (long long)blockIdx.x * kThreads + threadIdx.x; j < nvec; j += (long long)gridDim.x * kThreads) {
+        float4 xx = ld_last_use(xr + j * 4), vv = ld_last_use(vr + j * 4), gg = ld_last_use(gr + j * 4);
+        sgd4(xx, vv, gg, lr, mu, wd);
+        st_keep(vr + j * 4, vv);
+        st_keep(xr + j * 4, xx);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (long long i = nvec * 4; i < d; ++i) {
+            float xi = xr[i], vi = vr[i];
+            sgd1(xi, vi, gr[i], lr, mu, wd);
+            vr[i] = vi;
+            xr[i] = xi;
+        }
+    }
+}
+
+// Zero distances for the one-worker case (x_A == x_1).
+__global__ void zero_norms_kernel(float *norms_out, float *norms_stage, WsHeader *hdr) {
+    if (threadIdx.x == 0) {
+        norms_stage[0] = 0.f;
+        if (norms_out) norms_out[0] = 0.f;
+        hdr->status = DPPF_OK;
+        hdr->magic = 0;
+    }
+}
+
+// ---------------------------------------------------------------- host side
+
+struct DeviceInfo {
+    std::atomic<int> sms{0};
+    std::atomic<int> coop{-1};
+};
+DeviceInfo g_dev[64];   // immutable facts about each device, filled on first use
+
+int sm_count(int dev) {
+    int n = g_dev[dev].sms.load(std::memory_order_relaxed);
+    if (n == 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return -1;
+        g_dev[dev].sms.store(n, std::memory_order_relaxed);
+    }
+    return n;
+}
+
+bool coop_supported(int dev) {
+    int c = g_dev[dev].coop.load(std::memory_order_relaxed);
+    if (c < 0) {
+        if (cudaDeviceGetAttribute(&c, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) c = 0;
+        g_dev[dev].coop.store(c, std::memory_order_relaxed);
+    }
+    return c != 0;
+}
+
+int max_blocks_for(int M) { return M <= kMaxTemplateM ? kMaxBlocksSmallM : kMaxBlocksLargeM; }
+
+size_t norms_stage_offset(int M) {
+    size_t partial_bytes = (size_t)max_blocks_for(M) * (size_t)M * sizeof(double);
+    return kHeaderBytes + partial_bytes;
+}
+
+size_t workspace_bytes(int M) {
+    return norms_stage_offset(M) + (((size_t)M * sizeof(float) + 255) / 256) * 256;
+}
+
+bool finite_all(std::initializer_list<float> vals) {
+    for (float f : vals)
+        if (!std::isfinite(f)) return false;
+    return true;
+}
+
+bool aligned128(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 127u) == 0; }
+
+bool overlap(const void *a, size_t abytes, const void *b, size_t bbytes) {
+    uintptr_t pa = reinterpret_cast<uintptr_t>(a), pb = reinterpret_cast<uintptr_t>(b);
+    return pa < pb + bbytes && pb < pa + abytes;
+}
+
+int check_layout(const void *x, int M, int64_t d, int64_t ld) {
+    if (!x || M < 1 || M > DPPF_MAX_WORKERS || d < 1 || ld < d) return DPPF_ERR_INVALID_ARG;
+    if (ld > (int64_t)1 << 40) return DPPF_ERR_INVALID_ARG;
+    if (ld % 32 != 0 || !aligned128(x)) return DPPF_ERR_ALIGNMENT;
+    return DPPF_OK;
+}
+
+// Per-(M, kernel kind) resident blocks per SM, cached per device.
+std::atomic<int> g_occ[64][kMaxTemplateM + 1][2];
+
+template <typename K>
+int blocks_per_sm(K kernel, int dev, int M, int kind, size_t dyn_smem) {
+    int n = g_occ[dev][M][kind].load(std::memory_order_relaxed);
+    if (n == 0) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kThreads, dyn_smem) != cudaSuccess || n <= 0)
+            return -1;
+        g_occ[dev][M][kind].store(n, std::memory_order_relaxed);
+    }
+    return n;
+}
+
+template <int M>
+int launch_round_m(RoundArgs a, bool fused, int path, int dev, cudaStream_t s) {
+    constexpr int U = Tuning<M>::kUnroll;
+    const long long tile_vecs = (long long)kThreads * U;
+    long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
+    if (ntiles < 1) ntiles = 1;
+    const int sms = sm_count(dev);
+    if (sms <= 0) return DPPF_ERR_CUDA;
+
+    // Both schedules use the grid of the (larger) persistent kernel, so they split the
+    // sum of squares into the same per-block partials and give bit-identical results.
+    const int per_sm = fused ? blocks_per_sm(round_kernel<M, true>, dev, M, 1, 0)
+                             : blocks_per_sm(round_kernel<M, false>, dev, M, 0, 0);
+    if (per_sm <= 0) return DPPF_ERR_CUDA;
+    long long grid = (long long)sms * per_sm;
+    if (grid > ntiles) grid = ntiles;
+    if (grid > kMaxBlocksSmallM) grid = kMaxBlocksSmallM;
+
+    if (path == DPPF_PATH_COOPERATIVE && coop_supported(dev)) {
+        void *params[] = {&a};
+        const void *fn = fused ? (const void *)round_kernel<M, true> : (const void *)round_kernel<M, false>;
+        if (cudaLaunchCooperativeKernel(fn, dim3((unsigned)grid), dim3(kThreads), params, 0, s) != cudaSuccess) {
+            cudaGetLastError();
+            return DPPF_ERR_CUDA;
+        }
+        return DPPF_OK;
+    }
+    if (fused) distance_kernel<M, true><<<(unsigned)grid, kThreads, 0, s>>>(a);
+    else distance_kernel<M, false><<<(unsigned)grid, kThreads, 0, s>>>(a);
+    update_kernel<M><<<(unsigned)grid, kThreads, 0, s>>>(a, (int)grid);
+    if (cudaGetLastError() != cudaSuccess) return DPPF_ERR_CUDA;
+    return DPPF_OK;
+}
+
+int launch_round_generic(RoundArgs a, bool fused, int dev, cudaStream_t s) {
+    const int sms = sm_count(dev);
+    if (sms <= 0) return DPPF_ERR_CUDA;
+    long long ntiles = (a.nvec + kThreads - 1) / kThreads;
+    if (ntiles < 1) ntiles = 1;
+    long long grid = (long long)sms * 2;
+    if (grid > ntiles) grid = ntiles;
+    if (grid > kMaxBlocksLargeM) grid = kMaxBlocksLargeM;
+    const size_t smem_a = (size_t)kWarps * a.M * sizeof(float), smem_b = (size_t)a.M * sizeof(float);
+    if (smem_a > 48 * 1024) {
+        cudaError_t e = fused ? cudaFuncSetAttribute(distance_kernel_generic<true>,
+                                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_a)
+                              : cudaFuncSetAttribute(distance_kernel_generic<false>,
+                                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_a);
+        if (e != cudaSuccess) return DPPF_ERR_CUDA;
+    }
+    if (fused) distance_kernel_generic<true><<<(unsigned)grid, kThreads, smem_a, s>>>(a);
+    else distance_kernel_generic<false><<<(unsigned)grid, kThreads, smem_a, s>>>(a);
+    update_kernel_generic<<<(unsigned)grid, kThreads, smem_b, s>>>(a, (int)grid);
+    if (cudaGetLastError() != cudaSuccess) return DPPF_ERR_CUDA;
+    return DPPF_OK;
+}
+
+int launch_local_step(float *x, float *v, const float *g, int M, int64_t d, int64_t ld, float lr, float mu,
+                      float wd, int dev, cudaStream_t s) {
+    const int sms = sm_count(dev);
+    if (sms <= 0) return DPPF_ERR_CUDA;
+    const long long nvec = d / 4;
+    long long bx = (nvec + kThreads - 1) / kThreads;
+    const long long cap = ((long long)sms * 4 + M - 1) / M;   // about four blocks per SM over all rows
+    if (bx > cap) bx = cap;
+    if (bx < 1) bx = 1;
+    local_step_kernel<<<dim3((unsigned)bx, (unsigned)M), kThreads, 0, s>>>(x, v, g, d, ld, nvec, lr, mu, wd);
+    if (cudaGetLastError() != cudaSuccess) return DPPF_ERR_CUDA;
+    return DPPF_OK;
+}
+
+int resolve_path(int path, int M) {
+    if (M > kMaxTemplateM) return DPPF_PATH_TWO_KERNEL;
+    if (path == DPPF_PATH_AUTO) return DPPF_PATH_TWO_KERNEL;
+    return path;
+}
+
+int run_round(float *x, float *v, const float *g, int M, int64_t d, int64_t ld, float lr, float mu, float wd,
+              float alpha, float lambda, float *norms_out, void *ws, size_t ws_bytes, int path, bool fused,
+              cudaStream_t s) {
+    int rc = check_layout(x, M, d, ld);
+    if (rc != DPPF_OK) return rc;
+    if (path != DPPF_PATH_AUTO && path != DPPF_PATH_TWO_KERNEL && path != DPPF_PATH_COOPERATIVE)
+        return DPPF_ERR_INVALID_ARG;
+    if (!finite_all({alpha, lambda})) return DPPF_ERR_INVALID_ARG;
+    const size_t bytes = (size_t)M * (size_t)ld * sizeof(float);
+    if (fused) {
+        if ((rc = check_layout(v, M, d, ld)) != DPPF_OK) return rc;
+        if ((rc = check_layout(g, M, d, ld)) != DPPF_OK) return rc;
+        if (!finite_all({lr, mu, wd})) return DPPF_ERR_INVALID_ARG;
+        if (overlap(x, bytes, v, bytes) || overlap(x, bytes, g, bytes) || overlap(v, bytes, g, bytes)) return DPPF_ERR_INVALID_ARG;
+    }
+    if (!ws) return DPPF_ERR_INVALID_ARG;
+    if (!aligned128(ws)) return DPPF_ERR_ALIGNMENT;
+    if (ws_bytes < workspace_bytes(M)) return DPPF_ERR_WORKSPACE;
+    if (overlap(x, bytes, ws, workspace_bytes(M))) return DPPF_ERR_INVALID_ARG;
+
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DPPF_ERR_CUDA;
+
+    RoundArgs a;
+    a.x = x; a.v = v; a.g = g;
+    a.d = d; a.ld = ld; a.nvec = d / 4;
+    a.alpha = alpha; a.lambda = lambda; a.lr = lr; a.mu = mu; a.wd = wd;
+    a.norms_out = norms_out;
+    a.hdr = reinterpret_cast<WsHeader *>(ws);
+    a.partials = reinterpret_cast<double *>(static_cast<unsigned char *>(ws) + kHeaderBytes);
+    a.norms_stage = reinterpret_cast<float *>(static_cast<unsigned char *>(ws) + norms_stage_offset(M));
+    a.M = M;
+
+    if (M == 1) {   // x_A == x_1: distance 0, replica unchanged
+        if (fused && (rc = launch_local_step(x, v, g, M, d, ld, lr, mu, wd, dev, s)) != DPPF_OK) return rc;
+        zero_norms_kernel<<<1, 32, 0, s>>>(norms_out, a.norms_stage, a.hdr);
+        return cudaGetLastError() == cudaSuccess ? DPPF_OK : DPPF_ERR_CUDA;
+    }
+    path = resolve_path(path, M);
+    switch (M) {
+#define DPPF_CASE(MM) case MM: return launch_round_m<MM>(a, fused, path, dev, s);
+        DPPF_CASE(2) DPPF_CASE(3) DPPF_CASE(4) DPPF_CASE(5) DPPF_CASE(6) DPPF_CASE(7) DPPF_CASE(8)
+        DPPF_CASE(9) DPPF_CASE(10) DPPF_CASE(11) DPPF_CASE(12) DPPF_CASE(13) DPPF_CASE(14) DPPF_CASE(15)
+        DPPF_CASE(16)
+#undef DPPF_CASE
+        default: return launch_round_generic(a, fused, dev, s);
+    }
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------- C ABI
+
+extern "C" {
+
+size_t dppf_workspace_bytes(int M, int64_t d) {
+    if (M < 1 || M > DPPF_MAX_WORKERS || d < 1) return 0;
+    return workspace_bytes(M);
+}
+
+int dppf_consensus_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda, float *norms_out,
+                      void *ws, size_t ws_bytes, int path, void *cuda_stream) {
+    return run_round(x, nullptr, nullptr, M, d, ld, 0.f, 0.f, 0.f, alpha, lambda, norms_out, ws, ws_bytes, path,
+                     false, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int dppf_consensus(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda, float *norms_out, void *ws,
+                   size_t ws_bytes, void *cuda_stream) {
+    return dppf_consensus_ex(x, M, d, ld, alpha, lambda, norms_out, ws, ws_bytes, DPPF_PATH_AUTO, cuda_stream);
+}
+
+int dppf_local_step(float *x, float *v, const float *g, int M, int64_t d, int64_t ld, float lr, float momentum,
+                    float weight_decay, void *cuda_stream) {
+    int rc;
+    if ((rc = check_layout(x, M, d, ld)) != DPPF_OK) return rc;
+    if ((rc = check_layout(v, M, d, ld)) != DPPF_OK) return rc;
+    if ((rc = check_layout(g, M, d, ld)) != DPPF_OK) return rc;
+    if (!finite_all({lr, momentum, weight_decay})) return DPPF_ERR_INVALID_ARG;
+    const size_t bytes = (size_t)M * (size_t)ld * sizeof(float);
+    if (overlap(x, bytes, v, bytes) || overlap(x, bytes, g, bytes) || overlap(v, bytes, g, bytes)) return DPPF_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DPPF_ERR_CUDA;
+    return launch_local_step(x, v, g, M, d, ld, lr, momentum, weight_decay, dev,
+                             static_cast<cudaStream_t>(cuda_stream));
+}
+
+int dppf_local_step_and_consensus_ex(float *x, float *v, const float *g, int M, int64_t d, int64_t ld, float lr,
+                                     float momentum, float weight_decay, float alpha, float lambda,
+                                     float *norms_out, void *ws, size_t ws_bytes, int path, void *cuda_stream) {
+    return run_round(x, v, g, M, d, ld, lr, momentum, weight_decay, alpha, lambda, norms_out, ws, ws_bytes, path,
+                     true, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int dppf_local_step_and_consensus(float *x, float *v, const float *g, int M, int64_t d, int64_t ld, float lr,
+                                  float momentum, float weight_decay, float alpha, float lambda, float *norms_out,
+                                  void *ws, size_t ws_bytes, void *cuda_stream) {
+    return dppf_local_step_and_consensus_ex(x, v, g, M, d, ld, lr, momentum, weight_decay, alpha, lambda,
+                                            norms_out, ws, ws_bytes, DPPF_PATH_AUTO, cuda_stream);
+}
+
+int dppf_consensus_host(float *x_host, int M, int64_t d, int64_t ld, float alpha, float lambda, float *norms_host,
+                        float *x_dev, void *ws, size_t ws_bytes, void *cuda_stream) {
+    if (!x_host) return DPPF_ERR_INVALID_ARG;
+    int rc = check_layout(x_dev, M, d, ld);
+    if (rc != DPPF_OK) return rc;
+    if (!ws) return DPPF_ERR_INVALID_ARG;
+    if (!aligned128(ws)) return DPPF_ERR_ALIGNMENT;
+    if (ws_bytes < workspace_bytes(M)) return DPPF_ERR_WORKSPACE;
+    if (!finite_all({alpha, lambda})) return DPPF_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const size_t pitch = (size_t)ld * sizeof(float), width = (size_t)d * sizeof(float);
+    if (cudaMemcpy2DAsync(x_dev, pitch, x_host, pitch, width, (size_t)M, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return DPPF_ERR_CUDA;
+    rc = dppf_consensus(x_dev, M, d, ld, alpha, lambda, nullptr, ws, ws_bytes, cuda_stream);
+    if (rc != DPPF_OK) return rc;
+    if (cudaMemcpy2DAsync(x_host, pitch, x_dev, pitch, width, (size_t)M, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return DPPF_ERR_CUDA;
+    if (norms_host) {
+        const float *stage =
+            reinterpret_cast<const float *>(static_cast<unsigned char *>(ws) + norms_stage_offset(M));
+        if (cudaMemcpyAsync(norms_host, stage, (size_t)M * sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            return DPPF_ERR_CUDA;
+    }
+    return DPPF_OK;
+}
+
+int dppf_device_status(const void *ws, void *cuda_stream) {
+    if (!ws) return DPPF_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    int status = DPPF_OK;
+    if (cudaMemcpyAsync(&status, ws, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return DPPF_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return DPPF_ERR_CUDA;
+    return status;
+}
+
+const char *dppf_status_string(int status) {
+    switch (status) {
+        case DPPF_OK: return "DPPF_OK";
+        case DPPF_ERR_INVALID_ARG: return "DPPF_ERR_INVALID_ARG";
+        case DPPF_ERR_ALIGNMENT: return "DPPF_ERR_ALIGNMENT";
+        case DPPF_ERR_WORKSPACE: return "DPPF_ERR_WORKSPACE";
+        case DPPF_ERR_CUDA: return "DPPF_ERR_CUDA";
+        case DPPF_ERR_TIMEOUT: return "DPPF_ERR_TIMEOUT";
+        default: return "DPPF_ERR_UNKNOWN";
+    }
+}
+
+int dppf_launch_count(int M, int64_t d, int path, int fused) {
+    if (M < 1 || M > DPPF_MAX_WORKERS || d < 1) return 0;
+    if (M == 1) return fused ? 2 : 1;                       // [local step], zero norms
+    return resolve_path(path, M) == DPPF_PATH_COOPERATIVE ? 1 : 2;
+}
+
+}  // extern "C"

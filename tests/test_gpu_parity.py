@@ -1,0 +1,195 @@
+"""CUDA path vs the CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+
+from gpu_util import assert_pad_untouched, assert_parity, padded, require_gpu, same_bits, to_dev
+from paper_2507_20424_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+PATHS = {"two_kernel": 1, "cooperative": 2}
+
+
+def gpu_round(binding, x_np, d, alpha, lam, path):
+    import torch
+    M = x_np.shape[0]
+    x = to_dev(x_np)
+    norms = torch.full((M,), -1.0, device="cuda")
+    ws = binding.alloc_workspace(M, d)
+    binding.dppf_consensus(x, alpha, lam, norms_out=norms, ws=ws, d=d, path=path)
+    assert binding.dppf_device_status(ws) == binding.OK
+    return x.cpu().numpy(), norms.cpu().numpy()
+
+
+def random_replicas(M, d, seed, base=0.02, drift=1e-3):
+    rng = np.random.default_rng(seed)
+    x0 = rng.standard_normal(d) * base
+    return padded((x0[None, :] + rng.standard_normal((M, d)) * drift).astype(np.float32))
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 7, 8, 16, 17, 40])
+@pytest.mark.parametrize("d", [1, 3, 4, 31, 33, 127, 129, 4097, 100_003])
+def test_small_shapes(oracle, M, d, path):
+    _, binding = require_gpu()
+    x = random_replicas(M, d, seed=M * 1000 + d)
+    ref, r_ref = oracle.consensus(x, 0.1, 0.01, d=d)
+    got, r = gpu_round(binding, x, d, 0.1, 0.01, PATHS[path])
+    assert_parity(got, r, ref, r_ref, d)
+    assert_pad_untouched(got, d)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("name,d", [("C1", 1_048_576), ("C2", 3_000_017), ("C4", 5_000_005), ("C5", 2_000_003)])
+def test_workload_recipes_scaled(oracle, name, d, path):
+    """The benchmark recipes on vectors that span many tiles per block and a ragged tail."""
+    _, binding = require_gpu()
+    w = inputs.WORKLOADS[name].scaled(d)
+    x = inputs.replicas(w)
+    ref, r_ref = oracle.consensus(x, w.alpha, w.lam, d=w.d)
+    got, r = gpu_round(binding, x, w.d, w.alpha, w.lam, PATHS[path])
+    assert_parity(got, r, ref, r_ref, w.d)
+    assert_pad_untouched(got, w.d)
+
+
+@pytest.mark.parametrize("alpha,lam", [(1.0, 0.0), (0.5, 0.0), (0.0, 0.3), (0.9, 9.0), (0.5, 5.0), (0.05, 0.0)])
+def test_invariant_parameter_corners(oracle, alpha, lam):
+    _, binding = require_gpu()
+    x = random_replicas(4, 70_001, seed=5, base=0.5, drift=0.1)
+    ref, r_ref = oracle.consensus(x, alpha, lam, d=70_001)
+    got, r = gpu_round(binding, x, 70_001, alpha, lam, 1)
+    assert_parity(got, r, ref, r_ref, 70_001)
+    if alpha == 0.0:     # push only: every replica moves by exactly lambda
+        disp = np.linalg.norm(got[:, :70_001].astype(np.float64) - x[:, :70_001], axis=1)
+        np.testing.assert_allclose(disp, np.float32(lam), rtol=1e-5)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("M", [1, 2, 3, 5, 16, 24])
+def test_zero_distance_round_is_bit_exact(oracle, M, path):
+    _, binding = require_gpu()
+    w = inputs.WORKLOADS["C5"].scaled(1_000_003)
+    row = inputs.replicas(w, identical=True)[:1]
+    x = np.repeat(row, M, axis=0)
+    ref, r_ref = oracle.consensus(x, w.alpha, w.lam, d=w.d)
+    assert np.all(r_ref == 0.0) and same_bits(ref[:, :w.d], x[:, :w.d])
+    got, r = gpu_round(binding, x, w.d, w.alpha, w.lam, PATHS[path])
+    assert np.all(r == 0.0)
+    assert same_bits(got[:, :w.d], x[:, :w.d])
+    assert_pad_untouched(got, w.d)
+
+
+def test_mixed_zero_and_nonzero_distances(oracle):
+    """Two pairs of identical rows: no row is at zero distance, but deviations repeat exactly."""
+    _, binding = require_gpu()
+    base = random_replicas(2, 50_001, seed=9)
+    x = np.ascontiguousarray(base[[0, 0, 1, 1]])
+    ref, r_ref = oracle.consensus(x, 0.2, 0.05, d=50_001)
+    got, r = gpu_round(binding, x, 50_001, 0.2, 0.05, 1)
+    assert_parity(got, r, ref, r_ref, 50_001)
+    assert same_bits(got[0, :50_001], got[1, :50_001]) and same_bits(got[2, :50_001], got[3, :50_001])
+
+
+@pytest.mark.parametrize("M,d", [(4, 3_000_017), (8, 1_000_003), (16, 777_777), (20, 300_001)])
+def test_reproducible_and_schedule_independent(M, d):
+    """Same input -> same bits, run to run and across the two kernel schedules."""
+    _, binding = require_gpu()
+    x = random_replicas(M, d, seed=11)
+    a, ra = gpu_round(binding, x, d, 0.1, 0.01, 1)
+    b, rb = gpu_round(binding, x, d, 0.1, 0.01, 1)
+    c, rc = gpu_round(binding, x, d, 0.1, 0.01, 2)
+    assert same_bits(a[:, :d], b[:, :d]) and same_bits(ra, rb)
+    assert same_bits(a[:, :d], c[:, :d]) and same_bits(ra, rc)
+
+
+def test_norms_out_is_optional_and_iterated_rounds_follow_oracle(oracle):
+    import torch
+    _, binding = require_gpu()
+    d = 400_003
+    x_np = random_replicas(4, d, seed=13)
+    x = to_dev(x_np)
+    ws = binding.alloc_workspace(4, d)
+    ref = x_np
+    for k in range(20):
+        binding.dppf_consensus(x, 0.1, 0.005, norms_out=None, ws=ws, d=d, path=1 + k % 2)
+        ref, r_ref = oracle.consensus(ref, 0.1, 0.005, d=d)
+    norms = torch.zeros(4, device="cuda")
+    binding.dppf_consensus(x, 0.1, 0.005, norms_out=norms, ws=ws, d=d)
+    ref, r_ref = oracle.consensus(ref, 0.1, 0.005, d=d)
+    assert_parity(x.cpu().numpy(), norms.cpu().numpy(), ref, r_ref, d)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("M,d,tau", [(4, 1_000_003, 8), (2, 33, 3), (8, 200_001, 2), (16, 50_001, 2), (18, 40_003, 2), (1, 1000, 2)])
+def test_local_steps_then_fused_round(oracle, M, d, tau, path):
+    """tau-1 unfused local steps, then the last step fused with the round (x, v and r checked)."""
+    import torch
+    _, binding = require_gpu()
+    w = inputs.WORKLOADS["C3"].scaled(d)
+    w = type(w)(**{**w.__dict__, "M": M})
+    x_np, v_np = inputs.replicas(w), inputs.zeros_like_rows(w)
+    grads = [inputs.gradients(w, t) for t in range(tau)]
+    ref_x, ref_v, r_ref = oracle.local_steps_then_consensus(
+        x_np[:, :d], v_np[:, :d], [g[:, :d] for g in grads], w.lr, w.momentum, w.weight_decay, w.alpha, w.lam)
+    x, v = to_dev(x_np), to_dev(v_np)
+    ws = binding.alloc_workspace(M, d)
+    norms = torch.zeros(M, device="cuda")
+    for t in range(tau - 1):
+        binding.dppf_local_step(x, v, to_dev(grads[t]), w.lr, w.momentum, w.weight_decay, d=d)
+    g_last = to_dev(grads[-1])
+    binding.dppf_local_step_and_consensus(x, v, g_last, w.lr, w.momentum, w.weight_decay, w.alpha, w.lam,
+                                          norms_out=norms, ws=ws, d=d, path=PATHS[path])
+    assert binding.dppf_device_status(ws) == binding.OK
+    got_x, got_v = x.cpu().numpy(), v.cpu().numpy()
+    assert_parity(got_x, norms.cpu().numpy(), ref_x, r_ref, d)
+    verr = np.abs(got_v[:, :d].astype(np.float64) - ref_v[:, :d])
+    assert np.all(verr <= 1e-6 * (1 + np.abs(ref_v[:, :d])))
+    assert_pad_untouched(got_x, d), assert_pad_untouched(got_v, d)
+    assert same_bits(g_last.cpu().numpy()[:, :d], grads[-1][:, :d])     # gradients are read-only
+
+
+def test_fused_equals_unfused_sequence_bitwise():
+    _, binding = require_gpu()
+    w = inputs.WORKLOADS["C3"].scaled(300_001)
+    x_np, v_np, g_np = inputs.replicas(w), inputs.zeros_like_rows(w), inputs.gradients(w, 0)
+    x_np[:, :w.d] += inputs.gradients(w, 5)[:, :w.d]        # spread the replicas
+    ws = binding.alloc_workspace(w.M, w.d)
+    xa, va = to_dev(x_np), to_dev(v_np)
+    binding.dppf_local_step(xa, va, to_dev(g_np), w.lr, w.momentum, w.weight_decay, d=w.d)
+    binding.dppf_consensus(xa, w.alpha, w.lam, ws=ws, d=w.d)
+    xb, vb = to_dev(x_np), to_dev(v_np)
+    binding.dppf_local_step_and_consensus(xb, vb, to_dev(g_np), w.lr, w.momentum, w.weight_decay,
+                                          w.alpha, w.lam, ws=ws, d=w.d)
+    assert same_bits(xa.cpu().numpy()[:, :w.d], xb.cpu().numpy()[:, :w.d])
+    assert same_bits(va.cpu().numpy()[:, :w.d], vb.cpu().numpy()[:, :w.d])
+
+
+def test_host_resident_round(oracle):
+    import torch
+    _, binding = require_gpu()
+    d = 500_003
+    x_np = random_replicas(4, d, seed=17)
+    ref, r_ref = oracle.consensus(x_np, 0.1, 0.01, d=d)
+    x_host = torch.from_numpy(x_np.copy()).pin_memory()
+    norms_host = torch.zeros(4).pin_memory()
+    x_dev = binding.alloc_rows(4, d, fill=float("nan"))
+    ws = binding.alloc_workspace(4, d)
+    binding.dppf_consensus_host(x_host, 0.1, 0.01, norms_host, x_dev, ws, d=d)
+    torch.cuda.synchronize()
+    assert_parity(x_host.numpy(), norms_host.numpy(), ref, r_ref, d)
+    assert_pad_untouched(x_host.numpy(), d)
+
+
+def test_runs_on_a_side_stream(oracle):
+    import torch
+    _, binding = require_gpu()
+    d = 200_001
+    x_np = random_replicas(3, d, seed=19)
+    ref, r_ref = oracle.consensus(x_np, 0.3, 0.02, d=d)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        x = to_dev(x_np)
+        norms = torch.zeros(3, device="cuda")
+        binding.dppf_consensus(x, 0.3, 0.02, norms_out=norms, d=d)
+    s.synchronize()
+    assert_parity(x.cpu().numpy(), norms.cpu().numpy(), ref, r_ref, d)
