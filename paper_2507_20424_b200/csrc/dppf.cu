@@ -649,7 +649,7 @@ int launch_local_step(float *x, float *v, const float *g, int M, int64_t d, int6
 
 int resolve_path(int path, int M) {
     if (M > kMaxTemplateM) return DPPF_PATH_TWO_KERNEL;
-    if (path == DPPF_PATH_AUTO) return DPPF_PATH_TWO_KERNEL;
+    if (path == DPPF_PATH_AUTO) return DPPF_PATH_COOPERATIVE;   // one launch per round
     return path;
 }
 
