@@ -33,7 +33,7 @@ namespace cg = cooperative_groups;
 
 namespace {
 
-constexpr int kThreads = 256;            // threads per block, all kernels
+constexpr int kThreads = 256;            // threads per block: generic and local-step kernels
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxTemplateM = 16;        // worker counts with register-resident kernels
 constexpr int kMaxBlocksSmallM = 2048;   // partial-sum slots reserved per worker, M <= 16
@@ -142,12 +142,21 @@ __device__ __forceinline__ float coefficient(double S, float alpha, float lambda
 
 // ---------------------------------------------------------------- register-resident kernels (M <= 16)
 
+// Launch shape per worker count, from sweeps on B200.  The update pass mixes reads and
+// writes and is fastest with about 40-48 KB of loads in flight per SM; more outstanding
+// requests lower its DRAM efficiency, fewer cannot cover the latency.  The read-only distance
+// pass wants about twice that, which it gets from a deeper unroll on the same grid.
+//   bytes in flight per SM = kThreads * kBlocksPerSM * unroll * M * 16
 template <int M>
 struct Tuning {
-    // vectors per thread and tile iteration: keeps >= 64 bytes per row group in flight per thread
-    static constexpr int kUnroll = (M <= 2) ? 4 : (M <= 4) ? 2 : 1;
-    // blocks per SM the compiler must allow (register cap 64 / 85 / 128 per thread)
-    static constexpr int kMinBlocks = (M <= 4) ? 4 : (M <= 8) ? 3 : 2;
+    static constexpr int kThreads =
+        (M <= 2) ? 320 : (M == 3) ? 384 : (M == 4) ? 320 : (M == 5) ? 288 : (M == 6) ? 224 :
+        (M <= 8) ? 192 : (M == 9) ? 320 : (M == 10) ? 288 : (M <= 12) ? 256 : 224;
+    static constexpr int kBlocksPerSM = (M <= 8) ? 2 : 1;
+    static constexpr int kUnrollA = (M <= 2) ? 4 : (M <= 8) ? 2 : 1;      // distance pass
+    static constexpr int kUnrollFused = (M <= 2) ? 2 : 1;                 // distance pass with local step
+    static constexpr int kUnrollB = (M <= 2) ? 2 : 1;                     // update pass
+    static constexpr int kWarps = kThreads / 32;
 };
 
 // Scalar tail: columns 4*nvec .. d-1 (at most three), handled by one thread of block 0.
@@ -196,11 +205,12 @@ __device__ __forceinline__ void tail_update(const RoundArgs &a, const float *c) 
     }
 }
 
-// Distance pass body.  Tile t of the block = vectors [(t*U+u)*kThreads + tid], u < U.
+// Distance pass body.  Tile t of the block = vectors [(t*U+u)*T + tid], u < U.
 template <int M, bool kLocalStep>
-__device__ __forceinline__ void distance_pass(const RoundArgs &a, double *s_red /* [kWarps][M] */) {
-    constexpr int U = Tuning<M>::kUnroll;
-    const long long tile_vecs = (long long)kThreads * U;
+__device__ __forceinline__ void distance_pass(const RoundArgs &a, double *s_red /* [warps][M] */) {
+    constexpr int U = kLocalStep ? Tuning<M>::kUnrollFused : Tuning<M>::kUnrollA;
+    constexpr int T = Tuning<M>::kThreads;
+    const long long tile_vecs = (long long)T * U;
     const long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
     float acc[M];
 #pragma unroll
@@ -211,7 +221,7 @@ __device__ __forceinline__ void distance_pass(const RoundArgs &a, double *s_red 
         bool live[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const long long j = (t * U + u) * kThreads + threadIdx.x;
+            const long long j = (t * U + u) * T + threadIdx.x;
             live[u] = j < a.nvec;
             if (live[u]) {
 #pragma unroll
@@ -252,7 +262,7 @@ __device__ __forceinline__ void distance_pass(const RoundArgs &a, double *s_red 
     __syncthreads();
     if (threadIdx.x < M) {
         double s = 0.0;
-        for (int w = 0; w < kWarps; ++w) s += s_red[w * M + threadIdx.x];
+        for (int w = 0; w < Tuning<M>::kWarps; ++w) s += s_red[w * M + threadIdx.x];
         a.partials[(long long)blockIdx.x * M + threadIdx.x] = s;
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -269,7 +279,8 @@ __device__ __forceinline__ bool finalise(const RoundArgs &a, int M, int nblocks,
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0)
         *s_ok = (a.hdr->magic == kMagic && a.hdr->grid == nblocks && a.hdr->M == M) ? 1 : 0;
-    for (int m = warp; m < M; m += kWarps) {
+    const int nwarps = blockDim.x >> 5;
+    for (int m = warp; m < M; m += nwarps) {
         double s = 0.0;
         for (int b = lane; b < nblocks; b += 32) s += __ldcg(a.partials + (long long)b * M + m);
         s = warp_sum(s);
@@ -289,8 +300,9 @@ __device__ __forceinline__ bool finalise(const RoundArgs &a, int M, int nblocks,
 
 template <int M>
 __device__ __forceinline__ void update_pass(const RoundArgs &a, const float *s_c) {
-    constexpr int U = Tuning<M>::kUnroll;
-    const long long tile_vecs = (long long)kThreads * U;
+    constexpr int U = Tuning<M>::kUnrollB;
+    constexpr int T = Tuning<M>::kThreads;
+    const long long tile_vecs = (long long)T * U;
     const long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
     const float *c = s_c;
     if (ntiles > blockIdx.x) {
@@ -301,7 +313,7 @@ __device__ __forceinline__ void update_pass(const RoundArgs &a, const float *s_c
             bool live[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const long long j = (t * U + u) * kThreads + threadIdx.x;
+                const long long j = (t * U + u) * T + threadIdx.x;
                 live[u] = j < a.nvec;
                 if (live[u]) {
 #pragma unroll
@@ -311,7 +323,7 @@ __device__ __forceinline__ void update_pass(const RoundArgs &a, const float *s_c
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 if (live[u]) {
-                    const long long j = (t * U + u) * kThreads + threadIdx.x;
+                    const long long j = (t * U + u) * T + threadIdx.x;
                     const float4 ebar = shifted_mean<M>(xv[u]);
 #pragma unroll
                     for (int m = 0; m < M; ++m)
@@ -325,13 +337,13 @@ __device__ __forceinline__ void update_pass(const RoundArgs &a, const float *s_c
 }
 
 template <int M, bool kLocalStep>
-__global__ void __launch_bounds__(kThreads, Tuning<M>::kMinBlocks) distance_kernel(const RoundArgs a) {
-    __shared__ double s_red[kWarps * M];
+__global__ void __launch_bounds__(Tuning<M>::kThreads, Tuning<M>::kBlocksPerSM) distance_kernel(const RoundArgs a) {
+    __shared__ double s_red[Tuning<M>::kWarps * M];
     distance_pass<M, kLocalStep>(a, s_red);
 }
 
 template <int M>
-__global__ void __launch_bounds__(kThreads, Tuning<M>::kMinBlocks) update_kernel(const RoundArgs a, int nblocks_a) {
+__global__ void __launch_bounds__(Tuning<M>::kThreads, Tuning<M>::kBlocksPerSM) update_kernel(const RoundArgs a, int nblocks_a) {
     __shared__ float s_c[M];
     __shared__ int s_ok;
     if (!finalise(a, M, nblocks_a, s_c, &s_ok)) return;
@@ -341,8 +353,8 @@ __global__ void __launch_bounds__(kThreads, Tuning<M>::kMinBlocks) update_kernel
 // One persistent launch: distance pass, grid-wide barrier, update pass.  Launched with
 // cudaLaunchCooperativeKernel, which refuses the launch unless all blocks are co-resident.
 template <int M, bool kLocalStep>
-__global__ void __launch_bounds__(kThreads, Tuning<M>::kMinBlocks) round_kernel(const RoundArgs a) {
-    __shared__ double s_red[kWarps * M];
+__global__ void __launch_bounds__(Tuning<M>::kThreads, Tuning<M>::kBlocksPerSM) round_kernel(const RoundArgs a) {
+    __shared__ double s_red[Tuning<M>::kWarps * M];
     __shared__ float s_c[M];
     __shared__ int s_ok;
     distance_pass<M, kLocalStep>(a, s_red);
@@ -566,10 +578,10 @@ int check_layout(const void *x, int M, int64_t d, int64_t ld) {
 std::atomic<int> g_occ[64][kMaxTemplateM + 1][2];
 
 template <typename K>
-int blocks_per_sm(K kernel, int dev, int M, int kind, size_t dyn_smem) {
+int blocks_per_sm(K kernel, int dev, int M, int kind, int threads, size_t dyn_smem) {
     int n = g_occ[dev][M][kind].load(std::memory_order_relaxed);
     if (n == 0) {
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kThreads, dyn_smem) != cudaSuccess || n <= 0)
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, dyn_smem) != cudaSuccess || n <= 0)
             return -1;
         g_occ[dev][M][kind].store(n, std::memory_order_relaxed);
     }
@@ -578,18 +590,24 @@ int blocks_per_sm(K kernel, int dev, int M, int kind, size_t dyn_smem) {
 
 template <int M>
 int launch_round_m(RoundArgs a, bool fused, int path, int dev, cudaStream_t s) {
-    constexpr int U = Tuning<M>::kUnroll;
-    const long long tile_vecs = (long long)kThreads * U;
+    constexpr int T = Tuning<M>::kThreads;
+    // grid never exceeds the tile count of the pass with the largest tiles (the same bound
+    // with and without the fused local step, so both split the sums identically)
+    constexpr int u_ab = Tuning<M>::kUnrollA > Tuning<M>::kUnrollB ? Tuning<M>::kUnrollA : Tuning<M>::kUnrollB;
+    constexpr int u_max = u_ab > Tuning<M>::kUnrollFused ? u_ab : Tuning<M>::kUnrollFused;
+    const long long tile_vecs = (long long)T * u_max;
     long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
     if (ntiles < 1) ntiles = 1;
     const int sms = sm_count(dev);
     if (sms <= 0) return DPPF_ERR_CUDA;
 
-    // Both schedules use the grid of the (larger) persistent kernel, so they split the
-    // sum of squares into the same per-block partials and give bit-identical results.
-    const int per_sm = fused ? blocks_per_sm(round_kernel<M, true>, dev, M, 1, 0)
-                             : blocks_per_sm(round_kernel<M, false>, dev, M, 0, 0);
+    // Both schedules use the same grid (the tuned blocks per SM, never more than the
+    // persistent kernel can keep resident), so they split the sum of squares into the same
+    // per-block partials and give bit-identical results.
+    int per_sm = fused ? blocks_per_sm(round_kernel<M, true>, dev, M, 1, T, 0)
+                       : blocks_per_sm(round_kernel<M, false>, dev, M, 0, T, 0);
     if (per_sm <= 0) return DPPF_ERR_CUDA;
+    if (per_sm > Tuning<M>::kBlocksPerSM) per_sm = Tuning<M>::kBlocksPerSM;
     long long grid = (long long)sms * per_sm;
     if (grid > ntiles) grid = ntiles;
     if (grid > kMaxBlocksSmallM) grid = kMaxBlocksSmallM;
@@ -597,15 +615,15 @@ int launch_round_m(RoundArgs a, bool fused, int path, int dev, cudaStream_t s) {
     if (path == DPPF_PATH_COOPERATIVE && coop_supported(dev)) {
         void *params[] = {&a};
         const void *fn = fused ? (const void *)round_kernel<M, true> : (const void *)round_kernel<M, false>;
-        if (cudaLaunchCooperativeKernel(fn, dim3((unsigned)grid), dim3(kThreads), params, 0, s) != cudaSuccess) {
+        if (cudaLaunchCooperativeKernel(fn, dim3((unsigned)grid), dim3(T), params, 0, s) != cudaSuccess) {
             cudaGetLastError();
             return DPPF_ERR_CUDA;
         }
         return DPPF_OK;
     }
-    if (fused) distance_kernel<M, true><<<(unsigned)grid, kThreads, 0, s>>>(a);
-    else distance_kernel<M, false><<<(unsigned)grid, kThreads, 0, s>>>(a);
-    update_kernel<M><<<(unsigned)grid, kThreads, 0, s>>>(a, (int)grid);
+    if (fused) distance_kernel<M, true><<<(unsigned)grid, T, 0, s>>>(a);
+    else distance_kernel<M, false><<<(unsigned)grid, T, 0, s>>>(a);
+    update_kernel<M><<<(unsigned)grid, T, 0, s>>>(a, (int)grid);
     if (cudaGetLastError() != cudaSuccess) return DPPF_ERR_CUDA;
     return DPPF_OK;
 }
