@@ -122,6 +122,34 @@ int dppf_consensus_host(float *x_host, int M, int64_t d, int64_t ld, float alpha
                         void *cuda_stream);
 
 /*
+ * dppf_consensus with built-in scratch: for callers that cannot allocate.
+ * (The paper has no counterpart; this is a convenience of this library.)
+ *
+ * Some code that wants a round has no way to obtain a workspace: a plugin or callback that
+ * is handed device pointers by a host framework and must not allocate behind that
+ * framework's memory pool; a training process whose device memory was budgeted and handed
+ * out in full at start-up; a latency-critical loop in which allocation calls are banned
+ * because they can synchronise the device.  For those callers the per-block partial sums go
+ * to a fixed array inside the library's own device memory instead of a caller buffer.
+ *
+ *  - Same arguments, layout rules, result and return codes as dppf_consensus, minus ws and
+ *    ws_bytes.  The call makes no cudaMalloc/cudaFree and uses no allocating library routine.
+ *  - Limit: M <= DPPF_STATIC_MAX_WORKERS (16).  A larger M returns DPPF_ERR_WORKSPACE and
+ *    nothing is launched.  d is not limited.  The array is 262,656 bytes and every GPU
+ *    that loads the library keeps it until the process exits.
+ *  - The first call on each device looks up the array's device address (one
+ *    cudaGetSymbolAddress with that device current) and remembers it; make that first call
+ *    outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps whatever the previous call
+ *    left.  Nothing in it has to start at zero: every word a round reads it has written
+ *    earlier in the same round.  Two calls whose kernels can overlap on the GPU (different
+ *    streams without ordering) race on it; order them on one stream or with events.
+ */
+#define DPPF_STATIC_MAX_WORKERS 16
+int dppf_consensus_static(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
+                          float *norms_out, void *cuda_stream);
+
+/*
  * Synchronises `cuda_stream` and returns the status word the kernels keep in the
  * workspace header: DPPF_OK, or DPPF_ERR_WORKSPACE if the update pass found a
  * header that its distance pass did not write (workspace overwritten between the

@@ -19,7 +19,8 @@ OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range
 
 EXPORTS = ("dppf_workspace_bytes", "dppf_consensus", "dppf_consensus_ex", "dppf_local_step",
            "dppf_local_step_and_consensus", "dppf_local_step_and_consensus_ex",
-           "dppf_consensus_host", "dppf_device_status", "dppf_status_string", "dppf_launch_count")
+           "dppf_consensus_host", "dppf_device_status", "dppf_status_string", "dppf_launch_count",
+           "dppf_consensus_static")
 
 _lib = None
 
@@ -55,6 +56,8 @@ def load(rebuild_if_stale: bool = False) -> ctypes.CDLL:
     lib.dppf_local_step_and_consensus_ex.argtypes = [vp, vp, vp, i32, i64, i64, f32, f32, f32, f32, f32, vp, vp, sz, i32, vp]
     lib.dppf_consensus_host.argtypes = [vp, i32, i64, i64, f32, f32, vp, vp, vp, sz, vp]
     lib.dppf_device_status.argtypes = [vp, vp]
+    lib.dppf_consensus_static.argtypes = [vp, i32, i64, i64, f32, f32, vp, vp]
+    lib.dppf_consensus_static.restype = i32
     lib.dppf_status_string.argtypes = [i32]
     lib.dppf_status_string.restype = ctypes.c_char_p
     lib.dppf_launch_count.argtypes = [i32, i64, i32, i32]
@@ -118,6 +121,15 @@ def dppf_consensus(x, alpha, lam, norms_out=None, ws=None, d=None, path=PATH_AUT
                                   ws.data_ptr(), ws.numel(), int(path), _stream())
     _check(rc, "dppf_consensus")
     return ws
+
+
+def dppf_consensus_static(x, alpha, lam, norms_out=None, d=None):
+    """One round in place on ``x[M, ld]`` using the library's built-in scratch: no
+    workspace argument and no allocation anywhere in the call (M <= 16).  Calls that
+    may overlap on the GPU must be ordered by the caller; they share the scratch."""
+    M, d, ld = _dims(x, d)
+    rc = load().dppf_consensus_static(x.data_ptr(), M, d, ld, alpha, lam, _ptr(norms_out), _stream())
+    _check(rc, "dppf_consensus_static")
 
 
 def dppf_local_step(x, v, g, lr, momentum, weight_decay, d=None):

@@ -720,6 +720,32 @@ int run_round(float *x, float *v, const float *g, int M, int64_t d, int64_t ld, 
     }
 }
 
+// ---------------------------------------------------------------- built-in scratch
+// Scratch for dppf_consensus_static: one workspace image (header, per-block partial sums for
+// up to DPPF_STATIC_MAX_WORKERS workers, distance staging) that lives in the module's own
+// global memory.  Each GPU that loads the library carries these bytes until the process ends.
+constexpr size_t kStaticWsBytes =
+    kHeaderBytes + (size_t)kMaxBlocksSmallM * DPPF_STATIC_MAX_WORKERS * sizeof(double) + 256;
+static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
+
+// Device address of g_static_ws on each device.  In host code the name g_static_ws is only a
+// handle for the runtime, not an address a kernel can use; the real address comes from
+// cudaGetSymbolAddress, asked once per device while that device is current.
+std::atomic<void *> g_static_ws_addr[64];
+
+int static_ws_address(int dev, void **out) {
+    void *p = g_static_ws_addr[dev].load(std::memory_order_acquire);
+    if (p == nullptr) {
+        if (cudaGetSymbolAddress(&p, g_static_ws) != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return DPPF_ERR_CUDA;
+        }
+        g_static_ws_addr[dev].store(p, std::memory_order_release);
+    }
+    *out = p;
+    return DPPF_OK;
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------- C ABI
@@ -822,6 +848,21 @@ int dppf_launch_count(int M, int64_t d, int path, int fused) {
     if (M < 1 || M > DPPF_MAX_WORKERS || d < 1) return 0;
     if (M == 1) return fused ? 2 : 1;                       // [local step], zero norms
     return resolve_path(path, M) == DPPF_PATH_COOPERATIVE ? 1 : 2;
+}
+
+int dppf_consensus_static(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda, float *norms_out,
+                          void *cuda_stream) {
+    if (M > DPPF_STATIC_MAX_WORKERS) return DPPF_ERR_WORKSPACE;   // built-in scratch holds 16 workers at most
+    if (M < 1) return DPPF_ERR_INVALID_ARG;
+    if (workspace_bytes(M) > kStaticWsBytes) return DPPF_ERR_WORKSPACE;
+    int rc = check_layout(x, M, d, ld);      // reject bad arguments before any CUDA call
+    if (rc != DPPF_OK) return rc;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DPPF_ERR_CUDA;
+    void *ws = nullptr;
+    if ((rc = static_ws_address(dev, &ws)) != DPPF_OK) return rc;
+    return run_round(x, nullptr, nullptr, M, d, ld, 0.f, 0.f, 0.f, alpha, lambda, norms_out, ws, kStaticWsBytes,
+                     DPPF_PATH_AUTO, false, static_cast<cudaStream_t>(cuda_stream));
 }
 
 }  // extern "C"
