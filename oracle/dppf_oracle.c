@@ -18,8 +18,9 @@
  *
  * Readings where the paper is silent:
  *   - r_m == 0: the push direction is 0/0; no push is applied and the pull
- *     acts on a zero vector, so x_m is unchanged and r_m = 0 is reported
- *     (coefficient c_m = alpha).  No epsilon is added anywhere.
+ *     acts on a zero vector, so x_m is left exactly as it is (a plain copy,
+ *     which also keeps the sign of zeros) and r_m = 0 is reported.  No
+ *     epsilon is added anywhere.
  *   - local optimiser between rounds: Algorithm 1 prints plain SGD; the
  *     experiments use momentum 0.9 and weight decay without writing the
  *     recurrence.  The reading used is the standard coupled form
@@ -82,10 +83,14 @@ int dppf_oracle_consensus_f64(const double *x, int M, int64_t d, int64_t ld,
     average_f64(x, M, d, ld, A);
     distances_f64(x, M, d, ld, A, r_out);
     for (int m = 0; m < M; ++m) {
-        /* c_m = alpha - lambda / r_m ; zero distance: no push (see header) */
-        double c = (r_out[m] > 0.0) ? a - lam / r_out[m] : a;
+        /* c_m = alpha - lambda / r_m ; zero distance: replica unchanged (see header) */
         const double *xm = x + (int64_t)m * ld;
         float *om = x_out + (int64_t)m * ld_out;
+        if (!(r_out[m] > 0.0)) {
+            for (int64_t i = 0; i < d; ++i) om[i] = (float)xm[i];
+            continue;
+        }
+        double c = a - lam / r_out[m];
         for (int64_t i = 0; i < d; ++i)
             om[i] = (float)(xm[i] + (A[i] - xm[i]) * c);
     }
@@ -118,9 +123,13 @@ int dppf_oracle_consensus(const float *x, int M, int64_t d, int64_t ld,
         r_out[m] = sqrt(S);
     }
     for (int m = 0; m < M; ++m) {
-        double c = (r_out[m] > 0.0) ? a - lam / r_out[m] : a;
         const float *xm = x + (int64_t)m * ld;
         float *om = x_out + (int64_t)m * ld_out;
+        if (!(r_out[m] > 0.0)) {                 /* zero distance: replica unchanged */
+            for (int64_t i = 0; i < d; ++i) om[i] = xm[i];
+            continue;
+        }
+        double c = a - lam / r_out[m];
         for (int64_t i = 0; i < d; ++i) {
             double xi = (double)xm[i];
             om[i] = (float)(xi + (A[i] - xi) * c);
@@ -165,6 +174,10 @@ int dppf_oracle_consensus_two_step(const float *x, int M, int64_t d, int64_t ld,
             S1 += diff1 * diff1;
         }
         r_out[m] = sqrt(S0);                              /* pre-round distance */
+        if (!(r_out[m] > 0.0)) {                          /* zero distance: replica unchanged */
+            for (int64_t i = 0; i < d; ++i) om[i] = xm[i];
+            continue;
+        }
         double n1 = sqrt(S1);
         for (int64_t i = 0; i < d; ++i) {
             double push = (n1 > 0.0) ? lam * (y[i] - A[i]) / n1 : 0.0;
@@ -251,9 +264,13 @@ int dppf_oracle_consensus_blocked(const float *x, int M, int64_t d, int64_t ld,
     for (int t = 0; t < T; ++t) {
         int64_t lo = d * t / T, hi = d * (t + 1) / T;
         for (int m = 0; m < M; ++m) {
-            double c = (r_out[m] > 0.0) ? a - lam / r_out[m] : a;
             const float *xm = x + (int64_t)m * ld;
             float *om = x_out + (int64_t)m * ld_out;
+            if (!(r_out[m] > 0.0)) {             /* zero distance: replica unchanged */
+                for (int64_t i = lo; i < hi; ++i) om[i] = xm[i];
+                continue;
+            }
+            double c = a - lam / r_out[m];
             for (int64_t i = lo; i < hi; ++i) {
                 double xi = (double)xm[i];
                 om[i] = (float)(xi + (A[i] - xi) * c);

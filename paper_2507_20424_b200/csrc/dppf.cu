@@ -132,13 +132,17 @@ __device__ __forceinline__ double warp_sum(double a) {
     return a;   // butterfly: every lane holds the same bits
 }
 
-// Coefficient of the single-line update; zero distance -> no push (replica unchanged).
+// Coefficient c_m = alpha - lambda / r_m of the single-line update.  Zero distance: the push
+// direction is undefined and the pull acts on a zero vector, so the replica must stay as it
+// is, bit for bit (including the sign of zeros).  That case is signalled by a NaN coefficient,
+// which the update pass reads as "do not write this row".
 __device__ __forceinline__ float coefficient(double S, float alpha, float lambda, float *r_out) {
     double r = sqrt(S);
     *r_out = (float)r;
-    double c = (r > 0.0) ? (double)alpha - (double)lambda / r : (double)alpha;
-    return (float)c;
+    if (!(r > 0.0)) return __int_as_float(0x7fc00000);
+    return (float)((double)alpha - (double)lambda / r);
 }
+__device__ __forceinline__ bool row_is_written(float c) { return c == c; }
 
 // ---------------------------------------------------------------- register-resident kernels (M <= 16)
 
@@ -154,9 +158,15 @@ struct Tuning {
         (M <= 8) ? 192 : (M == 9) ? 320 : (M == 10) ? 288 : (M <= 12) ? 256 : 224;
     static constexpr int kBlocksPerSM = (M <= 8) ? 2 : 1;
     static constexpr int kUnrollA = (M <= 2) ? 4 : (M <= 8) ? 2 : 1;      // distance pass
-    static constexpr int kUnrollFused = (M <= 2) ? 2 : 1;                 // distance pass with local step
     static constexpr int kUnrollB = (M <= 2) ? 2 : 1;                     // update pass
+    // With the local step fused in, the distance pass moves five streams per row (x, v, g in,
+    // x, v out) and peaks at about half the resident threads (~60 KB of loads in flight per
+    // SM); the update pass of that launch doubles its unroll to keep its own 40-48 KB.
+    static constexpr int kBlocksPerSMFused = (kBlocksPerSM > 1) ? kBlocksPerSM / 2 : 1;
+    static constexpr int kUnrollFused = 1;
+    static constexpr int kUnrollBFused = kUnrollB * (kBlocksPerSM / kBlocksPerSMFused);
     static constexpr int kWarps = kThreads / 32;
+
 };
 
 // Scalar tail: columns 4*nvec .. d-1 (at most three), handled by one thread of block 0.
@@ -201,7 +211,8 @@ __device__ __forceinline__ void tail_update(const RoundArgs &a, const float *c) 
 #pragma unroll
         for (int m = 1; m < M; ++m) dv[m] = __fsub_rn(dv[m], ebar);
 #pragma unroll
-        for (int m = 0; m < M; ++m) a.x[m * a.ld + i] = __fmaf_rn(-c[m], dv[m], xs[m]);
+        for (int m = 0; m < M; ++m)
+            if (row_is_written(c[m])) a.x[m * a.ld + i] = __fmaf_rn(-c[m], dv[m], xs[m]);
     }
 }
 
@@ -224,20 +235,36 @@ __device__ __forceinline__ void distance_pass(const RoundArgs &a, double *s_red 
             const long long j = (t * U + u) * T + threadIdx.x;
             live[u] = j < a.nvec;
             if (live[u]) {
+                if (kLocalStep) {
+                    // Rows in groups of four: all loads of a group are issued before its first
+                    // store (x, v, g may not alias, but the compiler cannot know that and
+                    // would otherwise order every row's loads behind the previous row's stores).
+                    constexpr int G = 4;
 #pragma unroll
-                for (int m = 0; m < M; ++m) {
-                    const long long off = m * a.ld + j * 4;
-                    if (kLocalStep) {
-                        float4 xr = ld_last_use(a.x + off);
-                        float4 vr = ld_last_use(a.v + off);
-                        float4 gr = ld_last_use(a.g + off);
-                        sgd4(xr, vr, gr, a.lr, a.mu, a.wd);
-                        st_keep(a.v + off, vr);
-                        st_keep(a.x + off, xr);
-                        xv[u][m] = xr;
-                    } else {
-                        xv[u][m] = ld_keep(a.x + off);
+                    for (int m0 = 0; m0 < M; m0 += G) {
+                        float4 vv[G], gv[G];
+#pragma unroll
+                        for (int k = 0; k < G; ++k) {
+                            if (m0 + k < M) {
+                                const long long off = (m0 + k) * a.ld + j * 4;
+                                xv[u][m0 + k] = ld_last_use(a.x + off);
+                                vv[k] = ld_last_use(a.v + off);
+                                gv[k] = ld_last_use(a.g + off);
+                            }
+                        }
+#pragma unroll
+                        for (int k = 0; k < G; ++k) {
+                            if (m0 + k < M) {
+                                const long long off = (m0 + k) * a.ld + j * 4;
+                                sgd4(xv[u][m0 + k], vv[k], gv[k], a.lr, a.mu, a.wd);
+                                st_keep(a.v + off, vv[k]);
+                                st_keep(a.x + off, xv[u][m0 + k]);
+                            }
+                        }
                     }
+                } else {
+#pragma unroll
+                    for (int m = 0; m < M; ++m) xv[u][m] = ld_keep(a.x + m * a.ld + j * 4);
                 }
             }
         }
@@ -298,9 +325,8 @@ __device__ __forceinline__ bool finalise(const RoundArgs &a, int M, int nblocks,
     return *s_ok != 0;
 }
 
-template <int M>
+template <int M, int U>
 __device__ __forceinline__ void update_pass(const RoundArgs &a, const float *s_c) {
-    constexpr int U = Tuning<M>::kUnrollB;
     constexpr int T = Tuning<M>::kThreads;
     const long long tile_vecs = (long long)T * U;
     const long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
@@ -327,8 +353,9 @@ __device__ __forceinline__ void update_pass(const RoundArgs &a, const float *s_c
                     const float4 ebar = shifted_mean<M>(xv[u]);
 #pragma unroll
                     for (int m = 0; m < M; ++m)
-                        st_keep(a.x + m * a.ld + j * 4,
-                                apply4(xv[u][m], deviation(xv[u][m], xv[u][0], ebar, m), c[m]));
+                        if (row_is_written(c[m]))
+                            st_keep(a.x + m * a.ld + j * 4,
+                                    apply4(xv[u][m], deviation(xv[u][m], xv[u][0], ebar, m), c[m]));
                 }
             }
         }
@@ -337,30 +364,33 @@ __device__ __forceinline__ void update_pass(const RoundArgs &a, const float *s_c
 }
 
 template <int M, bool kLocalStep>
-__global__ void __launch_bounds__(Tuning<M>::kThreads, Tuning<M>::kBlocksPerSM) distance_kernel(const RoundArgs a) {
+__global__ void __launch_bounds__(Tuning<M>::kThreads, (kLocalStep ? Tuning<M>::kBlocksPerSMFused : Tuning<M>::kBlocksPerSM))
+distance_kernel(const RoundArgs a) {
     __shared__ double s_red[Tuning<M>::kWarps * M];
     distance_pass<M, kLocalStep>(a, s_red);
 }
 
-template <int M>
-__global__ void __launch_bounds__(Tuning<M>::kThreads, Tuning<M>::kBlocksPerSM) update_kernel(const RoundArgs a, int nblocks_a) {
+template <int M, bool kAfterLocalStep>
+__global__ void __launch_bounds__(Tuning<M>::kThreads, (kAfterLocalStep ? Tuning<M>::kBlocksPerSMFused : Tuning<M>::kBlocksPerSM))
+update_kernel(const RoundArgs a, int nblocks_a) {
     __shared__ float s_c[M];
     __shared__ int s_ok;
     if (!finalise(a, M, nblocks_a, s_c, &s_ok)) return;
-    update_pass<M>(a, s_c);
+    update_pass<M, (kAfterLocalStep ? Tuning<M>::kUnrollBFused : Tuning<M>::kUnrollB)>(a, s_c);
 }
 
 // One persistent launch: distance pass, grid-wide barrier, update pass.  Launched with
 // cudaLaunchCooperativeKernel, which refuses the launch unless all blocks are co-resident.
 template <int M, bool kLocalStep>
-__global__ void __launch_bounds__(Tuning<M>::kThreads, Tuning<M>::kBlocksPerSM) round_kernel(const RoundArgs a) {
+__global__ void __launch_bounds__(Tuning<M>::kThreads, (kLocalStep ? Tuning<M>::kBlocksPerSMFused : Tuning<M>::kBlocksPerSM))
+round_kernel(const RoundArgs a) {
     __shared__ double s_red[Tuning<M>::kWarps * M];
     __shared__ float s_c[M];
     __shared__ int s_ok;
     distance_pass<M, kLocalStep>(a, s_red);
     cg::this_grid().sync();
     if (!finalise(a, M, (int)gridDim.x, s_c, &s_ok)) return;
-    update_pass<M>(a, s_c);
+    update_pass<M, (kLocalStep ? Tuning<M>::kUnrollBFused : Tuning<M>::kUnrollB)>(a, s_c);
 }
 
 // ---------------------------------------------------------------- generic kernels (16 < M <= 1024)
@@ -465,7 +495,7 @@ __global__ void __launch_bounds__(kThreads) update_kernel_generic(const RoundArg
                 float *p = a.x + m * a.ld + j * 4;
                 float4 xr = (m == 0) ? x0 : *reinterpret_cast<const float4 *>(p);
                 float4 dv = (m == 0) ? make_float4(-ebar.x, -ebar.y, -ebar.z, -ebar.w) : sub4(sub4(xr, x0), ebar);
-                st_keep(p, apply4(xr, dv, s_c[m]));
+                if (row_is_written(s_c[m])) st_keep(p, apply4(xr, dv, s_c[m]));
             }
         }
     }
@@ -477,7 +507,7 @@ __global__ void __launch_bounds__(kThreads) update_kernel_generic(const RoundArg
             for (int m = M - 1; m >= 0; --m) {
                 float xi = a.x[m * a.ld + i];
                 float dv = (m == 0) ? -ebar : __fsub_rn(__fsub_rn(xi, x0s), ebar);
-                a.x[m * a.ld + i] = __fmaf_rn(-s_c[m], dv, xi);
+                if (row_is_written(s_c[m])) a.x[m * a.ld + i] = __fmaf_rn(-s_c[m], dv, xi);
             }
         }
     }
@@ -591,11 +621,10 @@ int blocks_per_sm(K kernel, int dev, int M, int kind, int threads, size_t dyn_sm
 template <int M>
 int launch_round_m(RoundArgs a, bool fused, int path, int dev, cudaStream_t s) {
     constexpr int T = Tuning<M>::kThreads;
-    // grid never exceeds the tile count of the pass with the largest tiles (the same bound
-    // with and without the fused local step, so both split the sums identically)
-    constexpr int u_ab = Tuning<M>::kUnrollA > Tuning<M>::kUnrollB ? Tuning<M>::kUnrollA : Tuning<M>::kUnrollB;
-    constexpr int u_max = u_ab > Tuning<M>::kUnrollFused ? u_ab : Tuning<M>::kUnrollFused;
-    const long long tile_vecs = (long long)T * u_max;
+    // grid never exceeds the tile count of the pass with the largest tiles
+    const int u_a = fused ? Tuning<M>::kUnrollFused : Tuning<M>::kUnrollA;
+    const int u_b = fused ? Tuning<M>::kUnrollBFused : Tuning<M>::kUnrollB;
+    const long long tile_vecs = (long long)T * (u_a > u_b ? u_a : u_b);
     long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
     if (ntiles < 1) ntiles = 1;
     const int sms = sm_count(dev);
@@ -607,7 +636,8 @@ int launch_round_m(RoundArgs a, bool fused, int path, int dev, cudaStream_t s) {
     int per_sm = fused ? blocks_per_sm(round_kernel<M, true>, dev, M, 1, T, 0)
                        : blocks_per_sm(round_kernel<M, false>, dev, M, 0, T, 0);
     if (per_sm <= 0) return DPPF_ERR_CUDA;
-    if (per_sm > Tuning<M>::kBlocksPerSM) per_sm = Tuning<M>::kBlocksPerSM;
+    const int tuned = fused ? Tuning<M>::kBlocksPerSMFused : Tuning<M>::kBlocksPerSM;
+    if (per_sm > tuned) per_sm = tuned;
     long long grid = (long long)sms * per_sm;
     if (grid > ntiles) grid = ntiles;
     if (grid > kMaxBlocksSmallM) grid = kMaxBlocksSmallM;
@@ -621,9 +651,13 @@ int launch_round_m(RoundArgs a, bool fused, int path, int dev, cudaStream_t s) {
         }
         return DPPF_OK;
     }
-    if (fused) distance_kernel<M, true><<<(unsigned)grid, T, 0, s>>>(a);
-    else distance_kernel<M, false><<<(unsigned)grid, T, 0, s>>>(a);
-    update_kernel<M><<<(unsigned)grid, T, 0, s>>>(a, (int)grid);
+    if (fused) {
+        distance_kernel<M, true><<<(unsigned)grid, T, 0, s>>>(a);
+        update_kernel<M, true><<<(unsigned)grid, T, 0, s>>>(a, (int)grid);
+    } else {
+        distance_kernel<M, false><<<(unsigned)grid, T, 0, s>>>(a);
+        update_kernel<M, false><<<(unsigned)grid, T, 0, s>>>(a, (int)grid);
+    }
     if (cudaGetLastError() != cudaSuccess) return DPPF_ERR_CUDA;
     return DPPF_OK;
 }

@@ -70,6 +70,7 @@ def test_zero_distance_round_is_bit_exact(oracle, M, path):
     _, binding = require_gpu()
     w = inputs.WORKLOADS["C5"].scaled(1_000_003)
     row = inputs.replicas(w, identical=True)[:1]
+    row[0, [5, 4096, 999_999]] = np.float32(-0.0)       # unchanged means the sign of zeros too
     x = np.repeat(row, M, axis=0)
     ref, r_ref = oracle.consensus(x, w.alpha, w.lam, d=w.d)
     assert np.all(r_ref == 0.0) and same_bits(ref[:, :w.d], x[:, :w.d])
@@ -148,20 +149,27 @@ def test_local_steps_then_fused_round(oracle, M, d, tau, path):
     assert same_bits(g_last.cpu().numpy()[:, :d], grads[-1][:, :d])     # gradients are read-only
 
 
-def test_fused_equals_unfused_sequence_bitwise():
+def test_fused_matches_unfused_sequence():
+    """Local step then round as two calls vs the fused call: the momentum buffers agree bit
+    for bit (same arithmetic); the replicas agree to rounding of the distances (the two
+    launches group the sum of squares into different per-block partials)."""
+    import torch
     _, binding = require_gpu()
-    w = inputs.WORKLOADS["C3"].scaled(300_001)
+    w = inputs.WORKLOADS["C3"].scaled(3_000_001)
     x_np, v_np, g_np = inputs.replicas(w), inputs.zeros_like_rows(w), inputs.gradients(w, 0)
     x_np[:, :w.d] += inputs.gradients(w, 5)[:, :w.d]        # spread the replicas
     ws = binding.alloc_workspace(w.M, w.d)
+    na, nb = torch.zeros(w.M, device="cuda"), torch.zeros(w.M, device="cuda")
     xa, va = to_dev(x_np), to_dev(v_np)
     binding.dppf_local_step(xa, va, to_dev(g_np), w.lr, w.momentum, w.weight_decay, d=w.d)
-    binding.dppf_consensus(xa, w.alpha, w.lam, ws=ws, d=w.d)
+    binding.dppf_consensus(xa, w.alpha, w.lam, norms_out=na, ws=ws, d=w.d)
     xb, vb = to_dev(x_np), to_dev(v_np)
     binding.dppf_local_step_and_consensus(xb, vb, to_dev(g_np), w.lr, w.momentum, w.weight_decay,
-                                          w.alpha, w.lam, ws=ws, d=w.d)
-    assert same_bits(xa.cpu().numpy()[:, :w.d], xb.cpu().numpy()[:, :w.d])
+                                          w.alpha, w.lam, norms_out=nb, ws=ws, d=w.d)
     assert same_bits(va.cpu().numpy()[:, :w.d], vb.cpu().numpy()[:, :w.d])
+    np.testing.assert_allclose(nb.cpu().numpy(), na.cpu().numpy(), rtol=1e-6)
+    xa_np, xb_np = xa.cpu().numpy()[:, :w.d], xb.cpu().numpy()[:, :w.d]
+    assert np.max(np.abs(xa_np.astype(np.float64) - xb_np)) <= 1e-8
 
 
 def test_host_resident_round(oracle):

@@ -131,8 +131,10 @@ def test_single_worker_unchanged(oracle):
 @pytest.mark.parametrize("M", [2, 3, 4, 7, 16])
 def test_identical_replicas_unchanged_bit_exact(oracle, M):
     row = rand_replicas(np.random.default_rng(5), 1, 777)
+    row[0, [3, 500]] = np.float32(-0.0)          # "unchanged" includes the sign of a zero
+    row[0, 7] = np.float32(0.0)
     x = np.repeat(row, M, axis=0)
-    for fn in (oracle.consensus, oracle.consensus_two_step):
+    for fn in (oracle.consensus, oracle.consensus_two_step, lambda *a: oracle.consensus_blocked(*a)[:2]):
         xp, r = fn(x, 0.2, 0.05)
         assert np.array_equal(xp.view(np.uint32), x.view(np.uint32))
         assert np.all(r == 0.0)
