@@ -47,7 +47,7 @@ typedef enum {
     DPPF_ERR_ALIGNMENT = 2,    /* base pointer not 128-byte aligned or ld % 32 != 0 */
     DPPF_ERR_WORKSPACE = 3,    /* ws_bytes < dppf_workspace_bytes(M, d) */
     DPPF_ERR_CUDA = 4,         /* a CUDA runtime call or launch failed */
-    DPPF_ERR_TIMEOUT = 5       /* reserved: a bounded device-side wait gave up */
+    DPPF_ERR_TIMEOUT = 5       /* device status only: a bounded wait on an async copy gave up */
 } dppf_status;
 
 /* Largest worker count handled (rows of x). */
@@ -57,6 +57,8 @@ typedef enum {
 #define DPPF_PATH_AUTO 0        /* library picks */
 #define DPPF_PATH_TWO_KERNEL 1  /* distance pass, then update pass, as two launches */
 #define DPPF_PATH_COOPERATIVE 2 /* one persistent cooperative launch with a grid-wide barrier */
+#define DPPF_PATH_STAGED 3      /* cooperative launch, rows staged through shared memory by bulk
+                                   async copies; what AUTO picks for dppf_consensus (M <= 16) */
 
 /*
  * Scratch size in bytes for a round on M replicas of length d (the per-block
@@ -74,8 +76,9 @@ size_t dppf_workspace_bytes(int M, int64_t d);
 int dppf_consensus(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
                    float *norms_out, void *ws, size_t ws_bytes, void *cuda_stream);
 
-/* Same, with an explicit kernel schedule (DPPF_PATH_*).  Both schedules give
- * bit-identical results. */
+/* Same, with an explicit kernel schedule (DPPF_PATH_*).  Every schedule is reproducible
+ * run to run; TWO_KERNEL and COOPERATIVE agree bit for bit, STAGED groups the sums of
+ * squares differently and may differ from them in the last bits of r_m. */
 int dppf_consensus_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
                       float *norms_out, void *ws, size_t ws_bytes, int path, void *cuda_stream);
 
@@ -151,9 +154,11 @@ int dppf_consensus_static(float *x, int M, int64_t d, int64_t ld, float alpha, f
 
 /*
  * Synchronises `cuda_stream` and returns the status word the kernels keep in the
- * workspace header: DPPF_OK, or DPPF_ERR_WORKSPACE if the update pass found a
+ * workspace header: DPPF_OK; DPPF_ERR_WORKSPACE if the update pass found a
  * header that its distance pass did not write (workspace overwritten between the
- * two), in which case x was left unchanged.  DPPF_ERR_CUDA if the stream failed.
+ * two), in which case x was left unchanged; DPPF_ERR_TIMEOUT if a bounded wait on an
+ * asynchronous copy gave up (x unchanged if that happened in the distance pass, partly
+ * updated otherwise).  DPPF_ERR_CUDA if the stream failed.
  */
 int dppf_device_status(const void *ws, void *cuda_stream);
 

@@ -14,7 +14,7 @@ import torch
 
 from . import build as _build
 
-PATH_AUTO, PATH_TWO_KERNEL, PATH_COOPERATIVE = 0, 1, 2
+PATH_AUTO, PATH_TWO_KERNEL, PATH_COOPERATIVE, PATH_STAGED = 0, 1, 2, 3
 OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
 
 EXPORTS = ("dppf_workspace_bytes", "dppf_consensus", "dppf_consensus_ex", "dppf_local_step",

@@ -7,7 +7,7 @@ from paper_2507_20424_b200 import inputs
 
 pytestmark = pytest.mark.gpu
 
-PATHS = {"two_kernel": 1, "cooperative": 2}
+PATHS = {"two_kernel": 1, "cooperative": 2, "staged": 3}
 
 
 def gpu_round(binding, x_np, d, alpha, lam, path):
@@ -93,7 +93,8 @@ def test_mixed_zero_and_nonzero_distances(oracle):
 
 @pytest.mark.parametrize("M,d", [(4, 3_000_017), (8, 1_000_003), (16, 777_777), (20, 300_001)])
 def test_reproducible_and_schedule_independent(M, d):
-    """Same input -> same bits, run to run and across the two kernel schedules."""
+    """Same input -> same bits run to run for every schedule; the two register schedules
+    also agree with each other bit for bit, the staged one to rounding of the distances."""
     _, binding = require_gpu()
     x = random_replicas(M, d, seed=11)
     a, ra = gpu_round(binding, x, d, 0.1, 0.01, 1)
@@ -101,6 +102,11 @@ def test_reproducible_and_schedule_independent(M, d):
     c, rc = gpu_round(binding, x, d, 0.1, 0.01, 2)
     assert same_bits(a[:, :d], b[:, :d]) and same_bits(ra, rb)
     assert same_bits(a[:, :d], c[:, :d]) and same_bits(ra, rc)
+    e, re_ = gpu_round(binding, x, d, 0.1, 0.01, 3)
+    f, rf = gpu_round(binding, x, d, 0.1, 0.01, 3)
+    assert same_bits(e[:, :d], f[:, :d]) and same_bits(re_, rf)
+    np.testing.assert_allclose(re_, ra, rtol=2e-6)
+    assert np.max(np.abs(e[:, :d].astype(np.float64) - a[:, :d])) <= 1e-8
 
 
 def test_norms_out_is_optional_and_iterated_rounds_follow_oracle(oracle):
@@ -112,7 +118,7 @@ def test_norms_out_is_optional_and_iterated_rounds_follow_oracle(oracle):
     ws = binding.alloc_workspace(4, d)
     ref = x_np
     for k in range(20):
-        binding.dppf_consensus(x, 0.1, 0.005, norms_out=None, ws=ws, d=d, path=1 + k % 2)
+        binding.dppf_consensus(x, 0.1, 0.005, norms_out=None, ws=ws, d=d, path=1 + k % 3)
         ref, r_ref = oracle.consensus(ref, 0.1, 0.005, d=d)
     norms = torch.zeros(4, device="cuda")
     binding.dppf_consensus(x, 0.1, 0.005, norms_out=norms, ws=ws, d=d)
