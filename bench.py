@@ -40,7 +40,7 @@ def parse_args():
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
     p.add_argument("--workload", default="C4")
     p.add_argument("--d", type=int, default=0, help="override the vector length (profiling on a smaller case)")
-    p.add_argument("--path", default="auto", choices=["auto", "two_kernel", "cooperative"])
+    p.add_argument("--path", default="auto", choices=["auto", "two_kernel", "cooperative", "staged"])
     p.add_argument("--e2e-steps", type=int, default=5)
     p.add_argument("--no-e2e", action="store_true")
     p.add_argument("--no-cpu-baseline", action="store_true")
@@ -58,18 +58,14 @@ def measured_peaks():
         return 6650.0, "fallback"
 
 
-def measured_traffic(w):
-    """DRAM bytes per launch from the committed ncu capture, scaled by replica bytes
-    (traffic grows in proportion to M*d once the replicas exceed L2); None if absent."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
-    try:
-        with open(path) as f:
-            t = json.load(f)
-        if not t.get("valid_for_current_kernel", False):
-            return None
-        return t["dram_bytes_per_replica_byte"] * w.M * w.d * 4
-    except Exception:
-        return None
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the single-pass
+# ncu capture of the full-size launch summarised in profiles/round_kernel_staged_M4.md.
+# Keyed by (workload, kernel); set an entry to None whenever that kernel changes.
+NCU_TRAFFIC = {("C4", 86_567_656, "staged"): 4.00e9}
+
+
+def measured_traffic(w, staged):
+    return NCU_TRAFFIC.get((w.name, w.d, "staged" if staged else "register"))
 
 
 def workload_of(args):
@@ -228,7 +224,11 @@ def run_ours(args):
     w = workload_of(args)
     seed = (inputs.DEFAULT_SEED if args.seed is None else args.seed) + rank
     path = {"auto": binding.PATH_AUTO, "two_kernel": binding.PATH_TWO_KERNEL,
-            "cooperative": binding.PATH_COOPERATIVE}[args.path]
+            "cooperative": binding.PATH_COOPERATIVE, "staged": binding.PATH_STAGED}[args.path]
+    staged = args.path == "staged" or (args.path == "auto" and w.M <= 8)
+    kernel_name = ("distance_kernel + update_kernel (one round)" if args.path == "two_kernel" else
+                   "round_kernel_staged (distance pass + grid barrier + update pass, one launch)" if staged else
+                   "round_kernel (distance pass + grid barrier + update pass, one launch)")
 
     # CPU baseline first (rank 0, N = 1 only): before any GPU work, so the OpenMP team is
     # created in a process that has not touched CUDA yet.
@@ -314,9 +314,8 @@ def run_ours(args):
                                         "schedule": args.path}),
                 "model_gbs_per_gpu": model_gbs, "frac_of_nominal_8tbs": model_gbs / NOMINAL_HBM_GBS,
                 "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                             "frac": achieved / peak, "traffic": measured_traffic(w),
-                             "kernel": "round_kernel (distance pass + grid barrier + update pass)"
-                             if launches_per_step == 1 else "distance_kernel + update_kernel (one round)",
+                             "frac": achieved / peak, "traffic": measured_traffic(w, staged),
+                             "kernel": kernel_name,
                              "algorithmic_bytes_per_launch": 3 * B, "peak_source": f"of {peak_src}"},
                 "clocks": clocks.summary(), "gpu_launches": K * launches_per_step,
                 "norms_last_round": [float(v) for v in norms.cpu().tolist()]}

@@ -58,7 +58,7 @@ typedef enum {
 #define DPPF_PATH_TWO_KERNEL 1  /* distance pass, then update pass, as two launches */
 #define DPPF_PATH_COOPERATIVE 2 /* one persistent cooperative launch with a grid-wide barrier */
 #define DPPF_PATH_STAGED 3      /* cooperative launch, rows staged through shared memory by bulk
-                                   async copies; what AUTO picks for dppf_consensus (M <= 16) */
+                                   async copies; what AUTO picks for dppf_consensus when M <= 8 */
 
 /*
  * Scratch size in bytes for a round on M replicas of length d (the per-block

@@ -394,7 +394,7 @@ round_kernel(const RoundArgs a) {
 }
 
 // ---------------------------------------------------------------- staged persistent kernel (default, M <= 16)
-// One block per SM keeps a ring of kStages shared-memory stages; a stage holds the same
+// One block per SM keeps a ring of up to kMaxStages shared-memory stages; a stage holds the same
 // column chunk of all M rows (about 32 KB).  One thread fills stages with 1-D bulk async
 // copies (cp.async.bulk, completion on an mbarrier); all threads then read the chunk from
 // shared memory.  Both passes run in this one cooperative launch:
@@ -410,16 +410,20 @@ round_kernel(const RoundArgs a) {
 
 constexpr int kStagedThreads = 256;
 constexpr int kStagedWarps = kStagedThreads / 32;
-constexpr int kStages = 6;
+constexpr int kMaxStages = 6;
 constexpr int kPrefetchA = 3;
 constexpr int kPrefetchB = 1;
 constexpr int kSpinLimit = 1 << 22;   // mbarrier try_wait polls before a wait gives up (~ a second)
 
 template <int M>
 struct StagedShape {
-    static constexpr int kChunk = ((8192 / M) / 128) * 128;        // columns per stage and row
+    // columns per stage and row: a stage of about 32 KB (40 KB measured best for M = 8)
+    static constexpr int kChunk = (M == 8) ? 1280 : ((8192 / M) / 128) * 128;
     static constexpr size_t kStageFloats = (size_t)M * kChunk;
+    static constexpr int kFit = (int)((200 * 1024) / (kStageFloats * sizeof(float)));
+    static constexpr int kStages = kFit < kMaxStages ? kFit : kMaxStages;
     static constexpr size_t kSmemBytes = (size_t)kStages * kStageFloats * sizeof(float);
+    static_assert(kStages > kPrefetchA, "ring must be deeper than the prefetch distance");
 };
 
 __device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -451,6 +455,7 @@ __device__ __forceinline__ void bulk_load(void *dst_smem, const void *src, unsig
 template <int M>
 __global__ void __launch_bounds__(kStagedThreads, 1) round_kernel_staged(const RoundArgs a) {
     constexpr int CH = StagedShape<M>::kChunk;
+    constexpr int kStages = StagedShape<M>::kStages;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     float *ring = reinterpret_cast<float *>(smem_raw);             // [kStages][M][CH]
     __shared__ unsigned long long full[kStages];
@@ -941,7 +946,8 @@ int launch_local_step(float *x, float *v, const float *g, int M, int64_t d, int6
 int resolve_path(int path, int M, bool fused) {
     if (M > kMaxTemplateM) return DPPF_PATH_TWO_KERNEL;
     if (fused && path == DPPF_PATH_STAGED) return DPPF_PATH_COOPERATIVE;   // no staged kernel with the local step
-    if (path == DPPF_PATH_AUTO) return fused ? DPPF_PATH_COOPERATIVE : DPPF_PATH_STAGED;   // one launch per round
+    // one launch per round; staging through shared memory pays off up to eight rows
+    if (path == DPPF_PATH_AUTO) return (fused || M > 8) ? DPPF_PATH_COOPERATIVE : DPPF_PATH_STAGED;
     return path;
 }
 
