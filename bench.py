@@ -208,6 +208,24 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------ replicas-only aggregation
+
+def max_over_ranks(ms, world, device=None):
+    """Slowest rank's elapsed time: the job is done when the last replica is."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(steps, world, elapsed_ms):
+    """Rounds per second over all ranks: every rank ran `steps` rounds on its own replica set."""
+    return world * steps / (elapsed_ms * 1e-3)
+
+
 # ------------------------------------------------------------------ CUDA arm
 
 def run_ours(args):
@@ -275,10 +293,7 @@ def run_ours(args):
     per_launch_ms = sum(ev[i].elapsed_time(ev[i + 1]) for i in range(K)) / K
     if binding.dppf_device_status(ws) != binding.OK:
         raise SystemExit("device status word reports an error")
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, "cuda")
     launches_per_step = binding.launch_count(w.M, w.d, path)
 
     # end-to-end: replicas live in pinned host memory; every step copies them in, runs the
@@ -295,17 +310,14 @@ def run_ours(args):
         e1.record()
         fence()
         e2e_ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e = {"value": world * args.e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+        e2e_ms = max_over_ranks(e2e_ms, world, "cuda")
+        e2e = {"value": whole_job_rate(args.e2e_steps, world, e2e_ms), "unit": UNIT,
                "h2d_bytes_per_step": B, "d2h_bytes_per_step": B + 4 * w.M, "steps": args.e2e_steps}
 
     if rank == 0:
         peak, peak_src = measured_peaks()
         achieved = 3.0 * B / (per_launch_ms * 1e-3) / 1e9
-        value = world * K / (total_ms * 1e-3)
+        value = whole_job_rate(K, world, total_ms)
         model_gbs = 3.0 * B * K / (total_ms * 1e-3) / 1e9
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
                 "warmup": max(3, args.warmup), "ms_per_step": total_ms / K, "higher_is_better": True,

@@ -1,0 +1,72 @@
+"""Host logic of the multi-GPU benchmark arm ("replicas only": N independent copies of the
+workload, no data-path collective), run as two gloo ranks on CPU."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+WORKER = r"""
+import os, sys, json
+sys.path.insert(0, sys.argv[1])
+import torch, torch.distributed as dist
+import bench
+from paper_2507_20424_b200 import inputs
+rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+dist.init_process_group("gloo")
+# every rank draws its own replica set (seed + rank), as the CUDA arm does
+w = inputs.WORKLOADS["C1"].scaled(1000)
+x = inputs.replicas(w, inputs.DEFAULT_SEED + rank)
+checksum = float(x[:, :w.d].astype("float64").sum())
+sums = [None] * world
+dist.all_gather_object(sums, checksum)
+# rank r pretends its timed region took (10 + 5 r) ms for 100 rounds
+ms = bench.max_over_ranks(10.0 + 5.0 * rank, world)
+rate = bench.whole_job_rate(100, world, ms)
+dist.barrier()
+if rank == 0:
+    print(json.dumps({"ms": ms, "rate": rate, "distinct_inputs": len(set(sums)) == world}))
+dist.destroy_process_group()
+"""
+
+
+def test_two_ranks_report_slowest_time_and_summed_rate(tmp_path):
+    script = tmp_path / "worker.py"
+    script.write_text(WORKER)
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+           "--master-addr", "127.0.0.1", "--master-port", "29533", str(script), ROOT]
+    run = subprocess.run(cmd, capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert run.returncode == 0, run.stderr[-2000:]
+    line = [l for l in run.stdout.splitlines() if l.startswith("{")][-1]
+    out = json.loads(line)
+    assert out["ms"] == 15.0                                   # the slower rank
+    assert out["rate"] == pytest.approx(2 * 100 / 0.015)       # both replicas' rounds count
+    assert out["distinct_inputs"]
+
+
+def test_single_rank_needs_no_process_group():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.max_over_ranks(12.5, 1) == 12.5
+    assert bench.whole_job_rate(1000, 1, 500.0) == 2000.0
+
+
+def test_reference_arm_prints_one_line_and_other_ranks_stay_silent():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2")
+    run = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
+                          "--warmup", "0"], capture_output=True, text=True, timeout=300, env=env, cwd=ROOT)
+    assert run.returncode == 0 and run.stdout.strip() == ""
+    env = dict(os.environ, RANK="0", WORLD_SIZE="2")
+    run = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "2",
+                          "--warmup", "1", "--workload", "C1", "--gpus", "2"],
+                         capture_output=True, text=True, timeout=300, env=env, cwd=ROOT)
+    assert run.returncode == 0, run.stderr[-2000:]
+    lines = [l for l in run.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1
+    out = json.loads(lines[0])
+    assert out["impl"] == "reference" and out["unit"] == "rounds/s" and out["value"] > 0
+    assert out["cpu_baseline"]["kind"] == "oracle" and out["cpu_baseline"]["cores"] >= 1
+    assert out["e2e"]["h2d_bytes_per_step"] == 0 and out["e2e"]["d2h_bytes_per_step"] == 0
