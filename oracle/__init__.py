@@ -56,6 +56,9 @@ def _load():
         lib.dppf_oracle_consensus_f64.argtypes = [f64p, i32, i64, i64, f32, f32, f32p, i64, f64p]
         lib.dppf_oracle_consensus_blocked.argtypes = common + [i32, ctypes.POINTER(i32)]
         lib.dppf_oracle_local_step_f64.argtypes = [f64p, f64p, f32p, i32, i64, i64, i64, f32, f32, f32]
+        lib.dppf_oracle_consensus_general.argtypes = [f32p, i32, i64, i64, f32, f32, f32p, i32, i32,
+                                                      f32p, i64, f64p, f64p]
+        lib.dppf_oracle_consensus_general.restype = i32
         for fn in (lib.dppf_oracle_consensus, lib.dppf_oracle_consensus_two_step,
                    lib.dppf_oracle_consensus_f64, lib.dppf_oracle_consensus_blocked,
                    lib.dppf_oracle_local_step_f64):
@@ -106,6 +109,29 @@ def consensus_blocked(x, alpha, lam, d=None, threads=0):
     out, r = _run(_load().dppf_oracle_consensus_blocked, x, d, alpha, lam,
                   extra=(int(threads), ctypes.byref(used)))
     return out, r, used.value
+
+
+def consensus_general(x, alpha, lam, weights=None, push_from="average", two_term=False, d=None):
+    """Algorithm 1 with a general consensus variable x_C = sum w_i x_i / sum w_i, the push
+    taken from x_A ("average") or from x_C ("consensus"), and optionally both terms of the
+    regulariser's gradient.  Returns (x_plus fp32, r fp64 = ||x_m - x_A||, n fp64 = ||y_m - P||)."""
+    M, ld = _check_2d(x, np.float32)
+    d = x.shape[1] if d is None else int(d)
+    out = np.array(x, copy=True, order="C")
+    r, n = np.zeros(M), np.zeros(M)
+    wp = None
+    if weights is not None:
+        w32 = np.ascontiguousarray(np.asarray(weights, dtype=np.float32))
+        if w32.shape != (M,):
+            raise ValueError("weights must have one entry per worker")
+        wp = _f32p(w32)
+    rc = _load().dppf_oracle_consensus_general(
+        _f32p(x), M, d, ld, np.float32(alpha), np.float32(lam), wp,
+        {"average": 0, "consensus": 1}[push_from], int(bool(two_term)),
+        _f32p(out), out.strides[0] // 4, _f64p(r), _f64p(n))
+    if rc != 0:
+        raise RuntimeError(f"oracle returned {rc}")
+    return out, r, n
 
 
 def local_steps_f64(x, v, grads, lr, momentum, weight_decay, d=None):

@@ -280,3 +280,102 @@ int dppf_oracle_consensus_blocked(const float *x, int M, int64_t d, int64_t ld,
     free(A); free(part);
     return 0;
 }
+
+/*
+ * General consensus round: Algorithm 1 with an arbitrary consensus variable and the
+ * optional second term of the regulariser's gradient.
+ *
+ *   x_A = (1/M) sum_i x_i                        (Algorithm 1, last line)
+ *   x_C = sum_i w_i x_i / sum_i w_i              ("any combination of worker parameters",
+ *                                                 Sec. 3; w = one-hot gives a leader, as in
+ *                                                 LSGD; w = NULL means x_C = x_A)
+ *   P   = x_A, or x_C when push_from_c != 0      (the remark on LSGD: the push may be
+ *                                                 redefined to oppose the leader)
+ *   pull    y_m = (1 - alpha) x_m + alpha x_C    (Algorithm 1, pull line)
+ *   u_m     = (y_m - P) / ||y_m - P||            (Algorithm 1, push line: direction of the
+ *                                                 pulled point from the reference point)
+ *   push    x_m+ = y_m + lambda u_m                            one term (Algorithm 1), or
+ *           x_m+ = y_m + lambda (u_m - (1/M) sum_j u_j)        both terms of step (a) of
+ *                                                 the regulariser-gradient equation in
+ *                                                 Sec. 5 with lambda = lambda_r / M
+ *
+ * Readings: x_A, x_C and P are the pre-round values for every worker (Jacobi, as in the
+ * proof of Theorem 1).  A worker whose pulled point coincides with P has no direction:
+ * u_m = 0 (no push for it, and it adds nothing to the mean direction).
+ * r_out[m]  = ||x_m - x_A||  before the round (the logged consensus distance),
+ * n_out[m]  = ||y_m - P||    (may be NULL).
+ * If every r_m is zero (identical replicas) x is copied unchanged.
+ */
+int dppf_oracle_consensus_general(const float *x, int M, int64_t d, int64_t ld,
+                                  float alpha, float lambda, const float *w,
+                                  int push_from_c, int two_term,
+                                  float *x_out, int64_t ld_out, double *r_out, double *n_out)
+{
+    if (!x || !x_out || !r_out || M < 1 || d < 1 || ld < d || ld_out < d) return 1;
+    double *A = (double *)malloc((size_t)d * sizeof(double));
+    double *C = (double *)malloc((size_t)d * sizeof(double));
+    double *ubar = (double *)calloc((size_t)d, sizeof(double));
+    double *nrm = (double *)malloc((size_t)M * sizeof(double));
+    if (!A || !C || !ubar || !nrm) { free(A); free(C); free(ubar); free(nrm); return 2; }
+    const double a = (double)alpha, lam = (double)lambda;
+    double wsum = 0.0;
+    for (int m = 0; m < M; ++m) wsum += w ? (double)w[m] : 1.0;
+    if (!(wsum != 0.0)) { free(A); free(C); free(ubar); free(nrm); return 1; }
+
+    for (int64_t i = 0; i < d; ++i) {
+        double s = 0.0, c = 0.0;
+        for (int m = 0; m < M; ++m) {
+            double xi = (double)x[(int64_t)m * ld + i];
+            s += xi;
+            c += (w ? (double)w[m] : 1.0) * xi;
+        }
+        A[i] = s / (double)M;
+        C[i] = c / wsum;
+    }
+    const double *P = push_from_c ? C : A;
+    int all_zero = 1;
+    for (int m = 0; m < M; ++m) {
+        const float *xm = x + (int64_t)m * ld;
+        double S = 0.0, N = 0.0;
+        for (int64_t i = 0; i < d; ++i) {
+            double xi = (double)xm[i];
+            double dr = xi - A[i];
+            S += dr * dr;
+            double y = (1.0 - a) * xi + a * C[i];
+            double dn = y - P[i];
+            N += dn * dn;
+        }
+        r_out[m] = sqrt(S);
+        nrm[m] = sqrt(N);
+        if (n_out) n_out[m] = nrm[m];
+        if (r_out[m] > 0.0) all_zero = 0;
+    }
+    if (all_zero) {
+        for (int m = 0; m < M; ++m)
+            for (int64_t i = 0; i < d; ++i) x_out[(int64_t)m * ld_out + i] = x[(int64_t)m * ld + i];
+        free(A); free(C); free(ubar); free(nrm);
+        return 0;
+    }
+    if (two_term) {
+        for (int m = 0; m < M; ++m) {
+            if (!(nrm[m] > 0.0)) continue;
+            const float *xm = x + (int64_t)m * ld;
+            for (int64_t i = 0; i < d; ++i) {
+                double y = (1.0 - a) * (double)xm[i] + a * C[i];
+                ubar[i] += (y - P[i]) / nrm[m];
+            }
+        }
+        for (int64_t i = 0; i < d; ++i) ubar[i] /= (double)M;
+    }
+    for (int m = 0; m < M; ++m) {
+        const float *xm = x + (int64_t)m * ld;
+        float *om = x_out + (int64_t)m * ld_out;
+        for (int64_t i = 0; i < d; ++i) {
+            double y = (1.0 - a) * (double)xm[i] + a * C[i];
+            double u = (nrm[m] > 0.0) ? (y - P[i]) / nrm[m] : 0.0;
+            om[i] = (float)(y + lam * (u - ubar[i]));      /* ubar is 0 unless two_term */
+        }
+    }
+    free(A); free(C); free(ubar); free(nrm);
+    return 0;
+}

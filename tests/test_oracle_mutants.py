@@ -25,6 +25,14 @@ MUTANTS = {
     "decay_operand": ("(double)gm[i] + wd * xm[i];", "(double)gm[i] + wd * vm[i];"),
     "descent_sign": ("xm[i] = xm[i] - eta * vm[i];", "xm[i] = xm[i] + eta * vm[i];"),
     "f64_round_coeff": ("(float)(xm[i] + (A[i] - xm[i]) * c)", "(float)(xm[i] + (A[i] - xm[i]) * a)"),
+    # general round
+    "g_push_reference": ("double dn = y - P[i];", "double dn = y - A[i];"),
+    "g_weight_norm": ("C[i] = c / wsum;", "C[i] = c;"),
+    "g_mean_direction": ("for (int64_t i = 0; i < d; ++i) ubar[i] /= (double)M;", ""),
+    "g_second_term_sign": ("lam * (u - ubar[i])", "lam * (u + ubar[i])"),
+    "g_pull_target": ("double y = (1.0 - a) * (double)xm[i] + a * C[i];\n            double u =",
+                      "double y = (1.0 - a) * (double)xm[i] + a * A[i];\n            double u ="),
+    "g_distance_reference": ("double dr = xi - A[i];", "double dr = xi - C[i];"),
 }
 
 
@@ -38,8 +46,11 @@ def test_pins_catch_mutant(tmp_path, name):
     assert old in src, f"mutation site for {name} not found"
     (dst / "dppf_oracle.c").write_text(src.replace(old, new))
     env = dict(os.environ, DPPF_ORACLE_PARENT=str(tmp_path))
-    run = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
-                          os.path.join(ROOT, "tests", "test_oracle_pins.py")],
+    files = [os.path.join(ROOT, "tests", "test_oracle_pins.py"),
+             os.path.join(ROOT, "tests", "test_oracle_general_pins.py")]
+    if name.startswith("g_"):
+        files.reverse()                      # the suite that should notice goes first (-x stops there)
+    run = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider", *files],
                          cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
     if name == "control_unchanged":          # the copy mechanism itself must not break the suite
         assert run.returncode == 0, run.stdout[-2000:]
