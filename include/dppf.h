@@ -83,6 +83,33 @@ int dppf_consensus_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float
                       float *norms_out, void *ws, size_t ws_bytes, int path, void *cuda_stream);
 
 /*
+ * General consensus round (Algorithm 1 with an arbitrary consensus variable; Sec. 5,
+ * step (a) of the regulariser-gradient equation; the remark on LSGD in the appendix):
+ *   x_C  = sum_m w_m x_m / sum_m w_m      weights_host: HOST fp32[M], NULL = all equal (x_C = x_A);
+ *                                         a one-hot vector makes one worker the leader
+ *   y_m  = (1 - alpha) x_m + alpha x_C    pull line of Algorithm 1
+ *   u_m  = (y_m - P) / ||y_m - P||        push line of Algorithm 1, P = x_A
+ *                                         (DPPF_PUSH_FROM_AVERAGE) or P = x_C
+ *                                         (DPPF_PUSH_FROM_CONSENSUS: push opposes the leader)
+ *   x_m <- y_m + lambda u_m                                     two_term == 0
+ *   x_m <- y_m + lambda (u_m - (1/M) sum_j u_j)                 two_term != 0: both terms of
+ *                                         the gradient of the relaxed Inverse-Mean-Valley
+ *                                         regulariser, lambda = lambda_r / M
+ * x_A, x_C and P are the pre-round values for every worker.  A worker whose pulled point
+ * equals P has no direction and is not pushed.  With weights_host == NULL, push from the
+ * average, two_term == 0 and alpha < 1 this is dppf_consensus.  Identical replicas are left
+ * untouched.  M <= 16.  norms_out (device fp32[M] or NULL) receives ||x_m - x_A|| before the
+ * round, push_norms_out (device fp32[M] or NULL) receives ||y_m - P||.  Workspace and layout
+ * rules as for dppf_consensus; same traffic (two reads and one write of x).
+ */
+#define DPPF_PUSH_FROM_AVERAGE 0
+#define DPPF_PUSH_FROM_CONSENSUS 1
+int dppf_consensus_general(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
+                           const float *weights_host, int push_from, int two_term,
+                           float *norms_out, float *push_norms_out, void *ws, size_t ws_bytes,
+                           void *cuda_stream);
+
+/*
  * One local optimiser step between rounds, in place, for all M workers
  * (Algorithm 1, the local update line; the experiments run SGD with momentum
  * and weight decay, whose recurrence the paper does not print -- the coupled

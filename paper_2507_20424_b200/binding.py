@@ -20,7 +20,7 @@ OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range
 EXPORTS = ("dppf_workspace_bytes", "dppf_consensus", "dppf_consensus_ex", "dppf_local_step",
            "dppf_local_step_and_consensus", "dppf_local_step_and_consensus_ex",
            "dppf_consensus_host", "dppf_device_status", "dppf_status_string", "dppf_launch_count",
-           "dppf_consensus_static")
+           "dppf_consensus_static", "dppf_consensus_general")
 
 _lib = None
 
@@ -56,6 +56,9 @@ def load(rebuild_if_stale: bool = False) -> ctypes.CDLL:
     lib.dppf_local_step_and_consensus_ex.argtypes = [vp, vp, vp, i32, i64, i64, f32, f32, f32, f32, f32, vp, vp, sz, i32, vp]
     lib.dppf_consensus_host.argtypes = [vp, i32, i64, i64, f32, f32, vp, vp, vp, sz, vp]
     lib.dppf_device_status.argtypes = [vp, vp]
+    lib.dppf_consensus_general.argtypes = [vp, i32, i64, i64, f32, f32, ctypes.POINTER(f32), i32, i32, vp, vp,
+                                           vp, sz, vp]
+    lib.dppf_consensus_general.restype = i32
     lib.dppf_consensus_static.argtypes = [vp, i32, i64, i64, f32, f32, vp, vp]
     lib.dppf_consensus_static.restype = i32
     lib.dppf_status_string.argtypes = [i32]
@@ -120,6 +123,27 @@ def dppf_consensus(x, alpha, lam, norms_out=None, ws=None, d=None, path=PATH_AUT
     rc = load().dppf_consensus_ex(x.data_ptr(), M, d, ld, alpha, lam, _ptr(norms_out),
                                   ws.data_ptr(), ws.numel(), int(path), _stream())
     _check(rc, "dppf_consensus")
+    return ws
+
+
+PUSH_FROM_AVERAGE, PUSH_FROM_CONSENSUS = 0, 1
+
+
+def dppf_consensus_general(x, alpha, lam, weights=None, push_from=PUSH_FROM_AVERAGE, two_term=False,
+                           norms_out=None, push_norms_out=None, ws=None, d=None):
+    """General round in place on ``x[M, ld]``: consensus variable from ``weights`` (host
+    sequence of M floats, None = plain average), push from x_A or x_C, optional second term."""
+    M, d, ld = _dims(x, d)
+    ws = alloc_workspace(M, d, x.device) if ws is None else ws
+    wp = None
+    if weights is not None:
+        if len(weights) != M:
+            raise ValueError("weights must have one entry per worker")
+        wp = (ctypes.c_float * M)(*[float(v) for v in weights])
+    rc = load().dppf_consensus_general(x.data_ptr(), M, d, ld, alpha, lam, wp, int(push_from), int(bool(two_term)),
+                                       _ptr(norms_out), _ptr(push_norms_out), ws.data_ptr(), ws.numel(),
+                                       _stream())
+    _check(rc, "dppf_consensus_general")
     return ws
 
 

@@ -85,6 +85,15 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert k(None, 4, 64, 64, 0.1, 0.01, None, X, WS, big, None) == b.ERR_INVALID_ARG
     assert k(V, 4, 64, 64, 0.1, 0.01, None, X + 4, WS, big, None) == b.ERR_ALIGNMENT
     assert lib.dppf_device_status(None, None) == b.ERR_INVALID_ARG
+    gen = lib.dppf_consensus_general
+    w_ok = (ctypes.c_float * 4)(1, 2, 3, 4)
+    w_zero = (ctypes.c_float * 4)(0, 0, 0, 0)
+    assert gen(None, 4, 64, 64, 0.1, 0.01, None, 0, 0, None, None, WS, big, None) == b.ERR_INVALID_ARG
+    assert gen(X, 17, 64, 64, 0.1, 0.01, None, 0, 0, None, None, WS, big, None) == b.ERR_INVALID_ARG
+    assert gen(X, 4, 64, 64, 0.1, 0.01, w_ok, 2, 0, None, None, WS, big, None) == b.ERR_INVALID_ARG
+    assert gen(X, 4, 64, 64, 0.1, 0.01, w_zero, 0, 0, None, None, WS, big, None) == b.ERR_INVALID_ARG
+    assert gen(X, 4, 64, 64, 0.1, 0.01, w_ok, 0, 1, None, None, WS, 16, None) == b.ERR_WORKSPACE
+    assert gen(X, 4, 60, 60, 0.1, 0.01, w_ok, 0, 1, None, None, WS, big, None) == b.ERR_ALIGNMENT
 
 
 def test_binding_refuses_cpu_tensors(lib):
