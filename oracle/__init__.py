@@ -59,6 +59,9 @@ def _load():
         lib.dppf_oracle_consensus_general.argtypes = [f32p, i32, i64, i64, f32, f32, f32p, i32, i32,
                                                       f32p, i64, f64p, f64p]
         lib.dppf_oracle_consensus_general.restype = i32
+        lib.dppf_oracle_adamw_step_f64.argtypes = [f64p, f64p, f64p, f32p, i32, i64, i64, i64,
+                                                   f32, f32, f32, f32, f32, i32]
+        lib.dppf_oracle_adamw_step_f64.restype = i32
         for fn in (lib.dppf_oracle_consensus, lib.dppf_oracle_consensus_two_step,
                    lib.dppf_oracle_consensus_f64, lib.dppf_oracle_consensus_blocked,
                    lib.dppf_oracle_local_step_f64):
@@ -153,6 +156,27 @@ def local_steps_f64(x, v, grads, lr, momentum, weight_decay, d=None):
         if rc != 0:
             raise RuntimeError(f"oracle returned {rc}")
     return x64, v64
+
+
+def adamw_steps_f64(x, m1, m2, grads, lr, beta1, beta2, eps, weight_decay, first_step=1, d=None):
+    """Apply ``len(grads)`` AdamW steps (step numbers first_step, first_step+1, ...) in fp64.
+    Returns the fp64 state (x, exp_avg, exp_avg_sq)."""
+    x64 = np.array(x, dtype=np.float64, order="C")
+    a64 = np.array(m1, dtype=np.float64, order="C")
+    b64 = np.array(m2, dtype=np.float64, order="C")
+    M, ld = _check_2d(x64, np.float64)
+    d = x64.shape[1] if d is None else int(d)
+    lib = _load()
+    for k, g in enumerate(grads):
+        Mg, ldg = _check_2d(g, np.float32)
+        if Mg != M or g.shape[1] < d:
+            raise ValueError("gradient shape mismatch")
+        rc = lib.dppf_oracle_adamw_step_f64(_f64p(x64), _f64p(a64), _f64p(b64), _f32p(g), M, d, ld, ldg,
+                                            np.float32(lr), np.float32(beta1), np.float32(beta2),
+                                            np.float32(eps), np.float32(weight_decay), int(first_step) + k)
+        if rc != 0:
+            raise RuntimeError(f"oracle returned {rc}")
+    return x64, a64, b64
 
 
 def consensus_f64(x64, alpha, lam, d=None):

@@ -379,3 +379,35 @@ int dppf_oracle_consensus_general(const float *x, int M, int64_t d, int64_t ld,
     free(A); free(C); free(ubar); free(nrm);
     return 0;
 }
+
+/*
+ * One AdamW local step on an fp64 state, in place.  The ViT experiments (appendix,
+ * "Experiments with ViT") train with AdamW, lr 5e-4, weight decay 0.01; the recurrence is
+ * not printed in the paper.  The reading used is the standard decoupled form:
+ *   x   <- x (1 - lr wd)
+ *   m   <- beta1 m + (1 - beta1) g
+ *   v   <- beta2 v + (1 - beta2) g^2
+ *   x   <- x - lr (m / (1 - beta1^t)) / ( sqrt(v / (1 - beta2^t)) + eps ),   t = step >= 1
+ */
+int dppf_oracle_adamw_step_f64(double *x, double *m1, double *m2, const float *g,
+                               int M, int64_t d, int64_t ld, int64_t ld_g,
+                               float lr, float beta1, float beta2, float eps, float weight_decay,
+                               int step)
+{
+    if (!x || !m1 || !m2 || !g || M < 1 || d < 1 || ld < d || ld_g < d || step < 1) return 1;
+    const double eta = (double)lr, b1 = (double)beta1, b2 = (double)beta2, e = (double)eps,
+                 wd = (double)weight_decay;
+    const double bc1 = 1.0 - pow(b1, (double)step), bc2 = 1.0 - pow(b2, (double)step);
+    for (int w = 0; w < M; ++w) {
+        double *xw = x + (int64_t)w * ld, *aw = m1 + (int64_t)w * ld, *bw = m2 + (int64_t)w * ld;
+        const float *gw = g + (int64_t)w * ld_g;
+        for (int64_t i = 0; i < d; ++i) {
+            double gi = (double)gw[i];
+            xw[i] = xw[i] * (1.0 - eta * wd);
+            aw[i] = b1 * aw[i] + (1.0 - b1) * gi;
+            bw[i] = b2 * bw[i] + (1.0 - b2) * gi * gi;
+            xw[i] = xw[i] - eta * (aw[i] / bc1) / (sqrt(bw[i] / bc2) + e);
+        }
+    }
+    return 0;
+}

@@ -25,6 +25,9 @@ MUTANTS = {
     "decay_operand": ("(double)gm[i] + wd * xm[i];", "(double)gm[i] + wd * vm[i];"),
     "descent_sign": ("xm[i] = xm[i] - eta * vm[i];", "xm[i] = xm[i] + eta * vm[i];"),
     "f64_round_coeff": ("(float)(xm[i] + (A[i] - xm[i]) * c)", "(float)(xm[i] + (A[i] - xm[i]) * a)"),
+    "adamw_decay": ("xw[i] = xw[i] * (1.0 - eta * wd);", "xw[i] = xw[i] * (1.0 - wd);"),
+    "adamw_second_moment": ("(1.0 - b2) * gi * gi;", "(1.0 - b2) * gi;"),
+    "adamw_bias": ("sqrt(bw[i] / bc2) + e", "sqrt(bw[i]) + e"),
     # general round
     "g_push_reference": ("double dn = y - P[i];", "double dn = y - A[i];"),
     "g_weight_norm": ("C[i] = c / wsum;", "C[i] = c;"),

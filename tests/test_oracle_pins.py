@@ -327,3 +327,45 @@ def test_local_steps_then_round_composes(oracle):
     a, l = float(np.float32(0.1)), float(np.float32(0.01))
     np.testing.assert_allclose(np.linalg.norm(xp - A, axis=1), np.abs((1 - a) * r + l), rtol=2e-6)
     np.testing.assert_allclose(r, np.linalg.norm(x64 - A, axis=1), rtol=1e-13)
+
+
+# ------------------------------------------------------------- AdamW local step
+
+def test_adamw_first_step_is_a_signed_step_of_size_lr(oracle):
+    # t = 1, zero moments: m/(1-b1) = g, v/(1-b2) = g^2  =>  x1 = x0 (1 - lr wd) - lr g / (|g| + eps)
+    rng = np.random.default_rng(21)
+    x0 = rand_replicas(rng, 2, 60)
+    g = f32(rng.standard_normal((2, 60)) * 1e-2)
+    z = np.zeros_like(x0)
+    lr, wd, eps = 5e-4, 0.01, 1e-8
+    x64, a64, b64 = oracle.adamw_steps_f64(x0, z, z, [g], lr, 0.9, 0.999, eps, wd)
+    lr32, wd32, eps32 = (float(np.float32(v)) for v in (lr, wd, eps))
+    g64 = g.astype(np.float64)
+    np.testing.assert_allclose(x64, x0.astype(np.float64) * (1 - lr32 * wd32) - lr32 * g64 / (np.abs(g64) + eps32),
+                               rtol=0, atol=1e-12)
+    np.testing.assert_allclose(a64, (1 - float(np.float32(0.9))) * g64, rtol=1e-14)
+    np.testing.assert_allclose(b64, (1 - float(np.float32(0.999))) * g64 ** 2, rtol=1e-14)
+
+
+def test_adamw_matches_library_adamw(oracle):
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(22)
+    M, d, tau = 3, 77, 6
+    lr, b1, b2, eps, wd = 5e-4, 0.9, 0.999, 1e-8, 0.01
+    x0 = rand_replicas(rng, M, d)
+    grads = [f32(rng.standard_normal((M, d)) * 1e-2) for _ in range(tau)]
+    p = torch.nn.Parameter(torch.tensor(x0, dtype=torch.float64))
+    f = lambda v: float(np.float32(v))
+    opt = torch.optim.AdamW([p], lr=f(lr), betas=(f(b1), f(b2)), eps=f(eps), weight_decay=f(wd), amsgrad=False)
+    for g in grads:
+        p.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+    z = np.zeros_like(x0)
+    x64, a64, b64 = oracle.adamw_steps_f64(x0, z, z, grads, lr, b1, b2, eps, wd)
+    np.testing.assert_allclose(x64, p.detach().numpy(), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(a64, opt.state[p]["exp_avg"].numpy(), rtol=1e-12, atol=1e-18)
+    np.testing.assert_allclose(b64, opt.state[p]["exp_avg_sq"].numpy(), rtol=1e-12, atol=1e-20)
+    # continuing from step 4 gives the same state as running straight through
+    xa, aa, ba = oracle.adamw_steps_f64(x0, z, z, grads[:3], lr, b1, b2, eps, wd)
+    xb, ab, bb = oracle.adamw_steps_f64(xa, aa, ba, grads[3:], lr, b1, b2, eps, wd, first_step=4)
+    assert np.array_equal(xb, x64) and np.array_equal(ab, a64) and np.array_equal(bb, b64)
