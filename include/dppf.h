@@ -137,6 +137,27 @@ int dppf_local_step_and_consensus_ex(float *x, float *v, const float *g, int M, 
                                      size_t ws_bytes, int path, void *cuda_stream);
 
 /*
+ * AdamW as the local optimiser (the paper's ViT runs: AdamW, lr 5e-4, weight decay 0.01;
+ * appendix, "Experiments with ViT").  The recurrence is not printed in the paper; the
+ * decoupled-weight-decay form is used, step = t >= 1 counting this step:
+ *   x <- x (1 - lr wd);  m <- beta1 m + (1 - beta1) g;  v <- beta2 v + (1 - beta2) g^2;
+ *   x <- x - lr (m / (1 - beta1^t)) / ( sqrt(v / (1 - beta2^t)) + eps )
+ * exp_avg (m) and exp_avg_sq (v) are device [M, ld] buffers, zero before step 1; g is read
+ * only; x, exp_avg, exp_avg_sq, g must not overlap; 0 <= beta < 1.
+ * dppf_adamw_step: the step alone, any M <= DPPF_MAX_WORKERS (7 x M d 4 bytes of traffic).
+ * dppf_adamw_step_and_consensus: the last step before a round fused with the round's
+ * distance pass (M <= 16; 9 x M d 4 bytes instead of 7 + 3): identical to dppf_adamw_step
+ * followed by dppf_consensus up to the grouping of the sums of squares.
+ */
+int dppf_adamw_step(float *x, float *exp_avg, float *exp_avg_sq, const float *g, int M, int64_t d,
+                    int64_t ld, float lr, float beta1, float beta2, float eps, float weight_decay,
+                    int step, void *cuda_stream);
+int dppf_adamw_step_and_consensus(float *x, float *exp_avg, float *exp_avg_sq, const float *g, int M,
+                                  int64_t d, int64_t ld, float lr, float beta1, float beta2, float eps,
+                                  float weight_decay, int step, float alpha, float lambda,
+                                  float *norms_out, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * Round on replicas that live in HOST memory (the arrangement the paper's
  * limitations section mentions: parameters kept off the accelerator).  Copies
  * x_host[M, ld] into the caller's device staging buffer x_dev[M, ld], runs

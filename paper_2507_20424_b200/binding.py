@@ -20,7 +20,8 @@ OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range
 EXPORTS = ("dppf_workspace_bytes", "dppf_consensus", "dppf_consensus_ex", "dppf_local_step",
            "dppf_local_step_and_consensus", "dppf_local_step_and_consensus_ex",
            "dppf_consensus_host", "dppf_device_status", "dppf_status_string", "dppf_launch_count",
-           "dppf_consensus_static", "dppf_consensus_general")
+           "dppf_consensus_static", "dppf_consensus_general",
+           "dppf_adamw_step", "dppf_adamw_step_and_consensus")
 
 _lib = None
 
@@ -56,6 +57,11 @@ def load(rebuild_if_stale: bool = False) -> ctypes.CDLL:
     lib.dppf_local_step_and_consensus_ex.argtypes = [vp, vp, vp, i32, i64, i64, f32, f32, f32, f32, f32, vp, vp, sz, i32, vp]
     lib.dppf_consensus_host.argtypes = [vp, i32, i64, i64, f32, f32, vp, vp, vp, sz, vp]
     lib.dppf_device_status.argtypes = [vp, vp]
+    lib.dppf_adamw_step.argtypes = [vp, vp, vp, vp, i32, i64, i64, f32, f32, f32, f32, f32, i32, vp]
+    lib.dppf_adamw_step.restype = i32
+    lib.dppf_adamw_step_and_consensus.argtypes = [vp, vp, vp, vp, i32, i64, i64, f32, f32, f32, f32, f32, i32,
+                                                  f32, f32, vp, vp, sz, vp]
+    lib.dppf_adamw_step_and_consensus.restype = i32
     lib.dppf_consensus_general.argtypes = [vp, i32, i64, i64, f32, f32, ctypes.POINTER(f32), i32, i32, vp, vp,
                                            vp, sz, vp]
     lib.dppf_consensus_general.restype = i32
@@ -176,6 +182,31 @@ def dppf_local_step_and_consensus(x, v, g, lr, momentum, weight_decay, alpha, la
         x.data_ptr(), v.data_ptr(), g.data_ptr(), M, d, ld, lr, momentum, weight_decay,
         alpha, lam, _ptr(norms_out), ws.data_ptr(), ws.numel(), int(path), _stream())
     _check(rc, "dppf_local_step_and_consensus")
+    return ws
+
+
+def _same_shape(x, others, d):
+    M, d, ld = _dims(x, d)
+    for t in others:
+        if _dims(t, d) != (M, d, ld):
+            raise ValueError("all buffers must share shape and row stride")
+    return M, d, ld
+
+
+def dppf_adamw_step(x, exp_avg, exp_avg_sq, g, lr, beta1, beta2, eps, weight_decay, step, d=None):
+    M, d, ld = _same_shape(x, (exp_avg, exp_avg_sq, g), d)
+    _check(load().dppf_adamw_step(x.data_ptr(), exp_avg.data_ptr(), exp_avg_sq.data_ptr(), g.data_ptr(), M, d, ld,
+                                  lr, beta1, beta2, eps, weight_decay, int(step), _stream()), "dppf_adamw_step")
+
+
+def dppf_adamw_step_and_consensus(x, exp_avg, exp_avg_sq, g, lr, beta1, beta2, eps, weight_decay, step,
+                                  alpha, lam, norms_out=None, ws=None, d=None):
+    M, d, ld = _same_shape(x, (exp_avg, exp_avg_sq, g), d)
+    ws = alloc_workspace(M, d, x.device) if ws is None else ws
+    rc = load().dppf_adamw_step_and_consensus(
+        x.data_ptr(), exp_avg.data_ptr(), exp_avg_sq.data_ptr(), g.data_ptr(), M, d, ld, lr, beta1, beta2, eps,
+        weight_decay, int(step), alpha, lam, _ptr(norms_out), ws.data_ptr(), ws.numel(), _stream())
+    _check(rc, "dppf_adamw_step_and_consensus")
     return ws
 
 

@@ -393,6 +393,146 @@ round_kernel(const RoundArgs a) {
     update_pass<M, (kLocalStep ? Tuning<M>::kUnrollBFused : Tuning<M>::kUnrollB)>(a, s_c);
 }
 
+// ---------------------------------------------------------------- AdamW local step (fused and stand-alone)
+// The ViT runs of the paper train with AdamW (lr 5e-4, weight decay 0.01).  Decoupled form:
+//   x <- x (1 - lr wd);  m <- m + (1 - b1)(g - m);  v <- b2 v + (1 - b2) g^2;
+//   x <- x - [lr / (1 - b1^t)] m / ( sqrt(v) / sqrt(1 - b2^t) + eps )
+// The step-dependent factors are formed on the host in double and passed as floats.
+
+struct AdamArgs {
+    float *m1;   // exp_avg      [M, ld]
+    float *m2;   // exp_avg_sq   [M, ld]
+    const float *g;
+    float decay, one_minus_b1, b2, one_minus_b2, step_size, inv_sqrt_bc2, eps;
+};
+
+__device__ __forceinline__ void adamw1(float &x, float &m1, float &m2, float g, const AdamArgs &p) {
+    x = __fmul_rn(x, p.decay);
+    m1 = __fmaf_rn(p.one_minus_b1, __fsub_rn(g, m1), m1);
+    m2 = __fmaf_rn(p.b2, m2, __fmul_rn(p.one_minus_b2, __fmul_rn(g, g)));
+    const float denom = __fmaf_rn(__fsqrt_rn(m2), p.inv_sqrt_bc2, p.eps);
+    x = __fmaf_rn(-p.step_size, __fdiv_rn(m1, denom), x);
+}
+__device__ __forceinline__ void adamw4(float4 &x, float4 &m1, float4 &m2, float4 g, const AdamArgs &p) {
+    adamw1(x.x, m1.x, m2.x, g.x, p);
+    adamw1(x.y, m1.y, m2.y, g.y, p);
+    adamw1(x.z, m1.z, m2.z, g.z, p);
+    adamw1(x.w, m1.w, m2.w, g.w, p);
+}
+
+// Distance pass with the AdamW step applied first; leaves the same partial sums and header
+// as distance_kernel, so update_kernel<M, false> completes the round.  Measured best with
+// the plain round's residency and two rows of loads in flight per thread.
+template <int M>
+__global__ void __launch_bounds__(Tuning<M>::kThreads, Tuning<M>::kBlocksPerSM)
+adamw_distance_kernel(const RoundArgs a, const AdamArgs p) {
+    constexpr int T = Tuning<M>::kThreads;
+    constexpr int G = 2;                               // rows whose loads are issued together
+    __shared__ double s_red[Tuning<M>::kWarps * M];
+    const long long ntiles = (a.nvec + T - 1) / T;
+    float acc[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) acc[m] = 0.f;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        const long long j = t * T + threadIdx.x;
+        if (j < a.nvec) {
+            float4 xv[M];
+#pragma unroll
+            for (int m0 = 0; m0 < M; m0 += G) {
+                float4 av[G], bv[G], gv[G];
+#pragma unroll
+                for (int k = 0; k < G; ++k) {
+                    if (m0 + k < M) {
+                        const long long off = (m0 + k) * a.ld + j * 4;
+                        xv[m0 + k] = ld_last_use(a.x + off);
+                        av[k] = ld_last_use(p.m1 + off);
+                        bv[k] = ld_last_use(p.m2 + off);
+                        gv[k] = ld_last_use(p.g + off);
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < G; ++k) {
+                    if (m0 + k < M) {
+                        const long long off = (m0 + k) * a.ld + j * 4;
+                        adamw4(xv[m0 + k], av[k], bv[k], gv[k], p);
+                        st_keep(p.m1 + off, av[k]);
+                        st_keep(p.m2 + off, bv[k]);
+                        st_keep(a.x + off, xv[m0 + k]);
+                    }
+                }
+            }
+            const float4 ebar = shifted_mean<M>(xv);
+#pragma unroll
+            for (int m = 0; m < M; ++m) acc[m] = sq_acc(acc[m], deviation(xv[m], xv[0], ebar, m));
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {          // scalar tail columns
+        const float inv_m = 1.0f / (float)M;
+        for (long long i = a.nvec * 4; i < a.d; ++i) {
+            float xs[M];
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                const long long off = m * a.ld + i;
+                float xi = a.x[off], ai = p.m1[off], bi = p.m2[off];
+                adamw1(xi, ai, bi, p.g[off], p);
+                p.m1[off] = ai;
+                p.m2[off] = bi;
+                a.x[off] = xi;
+                xs[m] = xi;
+            }
+            float esum = 0.f;
+#pragma unroll
+            for (int m = 1; m < M; ++m) { xs[m] = __fsub_rn(xs[m], xs[0]); esum = __fadd_rn(esum, xs[m]); }
+            const float ebar = __fmul_rn(esum, inv_m);
+            acc[0] = __fmaf_rn(ebar, ebar, acc[0]);
+#pragma unroll
+            for (int m = 1; m < M; ++m) { float dv = __fsub_rn(xs[m], ebar); acc[m] = __fmaf_rn(dv, dv, acc[m]); }
+        }
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+        double sum = warp_sum((double)acc[m]);
+        if (lane == 0) s_red[warp * M + m] = sum;
+    }
+    __syncthreads();
+    if (threadIdx.x < M) {
+        double sum = 0.0;
+        for (int w = 0; w < Tuning<M>::kWarps; ++w) sum += s_red[w * M + threadIdx.x];
+        a.partials[(long long)blockIdx.x * M + threadIdx.x] = sum;
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        a.hdr->status = DPPF_OK;
+        a.hdr->magic = kMagic;
+        a.hdr->grid = (int)gridDim.x;
+        a.hdr->M = M;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) adamw_step_kernel(float *x, const AdamArgs p, long long d, long long ld,
+                                                              long long nvec) {
+    const long long row = (long long)blockIdx.y * ld;
+    for (long long j = (long long)blockIdx.x * kThreads + threadIdx.x; j < nvec; j += (long long)gridDim.x * kThreads) {
+        const long long off = row + j * 4;
+        float4 xx = ld_last_use(x + off), aa = ld_last_use(p.m1 + off), bb = ld_last_use(p.m2 + off),
+               gg = ld_last_use(p.g + off);
+        adamw4(xx, aa, bb, gg, p);
+        st_keep(p.m1 + off, aa);
+        st_keep(p.m2 + off, bb);
+        st_keep(x + off, xx);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (long long i = nvec * 4; i < d; ++i) {
+            const long long off = row + i;
+            float xi = x[off], ai = p.m1[off], bi = p.m2[off];
+            adamw1(xi, ai, bi, p.g[off], p);
+            p.m1[off] = ai;
+            p.m2[off] = bi;
+            x[off] = xi;
+        }
+    }
+}
+
 // ---------------------------------------------------------------- staged persistent kernel (default, M <= 16)
 // One block per SM keeps a ring of up to kMaxStages shared-memory stages; a stage holds the same
 // column chunk of all M rows (about 32 KB).  One thread fills stages with 1-D bulk async
@@ -1362,6 +1502,67 @@ int launch_general_m(const GeneralArgs &a, int dev, cudaStream_t s) {
     return DPPF_OK;
 }
 
+
+// ---------------------------------------------------------------- AdamW: host side
+int make_adam_args(float *m1, float *m2, const float *g, float lr, float beta1, float beta2, float eps, float wd,
+                   int step, AdamArgs *out) {
+    if (!finite_all({lr, beta1, beta2, eps, wd}) || step < 1) return DPPF_ERR_INVALID_ARG;
+    if (!(beta1 >= 0.f && beta1 < 1.f && beta2 >= 0.f && beta2 < 1.f)) return DPPF_ERR_INVALID_ARG;
+    const double bc1 = 1.0 - std::pow((double)beta1, (double)step);
+    const double bc2 = 1.0 - std::pow((double)beta2, (double)step);
+    out->m1 = m1; out->m2 = m2; out->g = g;
+    out->decay = (float)(1.0 - (double)lr * (double)wd);
+    out->one_minus_b1 = (float)(1.0 - (double)beta1);
+    out->b2 = beta2;
+    out->one_minus_b2 = (float)(1.0 - (double)beta2);
+    out->step_size = (float)((double)lr / bc1);
+    out->inv_sqrt_bc2 = (float)(1.0 / std::sqrt(bc2));
+    out->eps = eps;
+    return DPPF_OK;
+}
+
+int check_adam_buffers(const float *x, const float *m1, const float *m2, const float *g, int M, int64_t d, int64_t ld) {
+    int rc;
+    if ((rc = check_layout(x, M, d, ld)) != DPPF_OK) return rc;
+    if ((rc = check_layout(m1, M, d, ld)) != DPPF_OK) return rc;
+    if ((rc = check_layout(m2, M, d, ld)) != DPPF_OK) return rc;
+    if ((rc = check_layout(g, M, d, ld)) != DPPF_OK) return rc;
+    const size_t bytes = (size_t)M * (size_t)ld * sizeof(float);
+    const void *bufs[4] = {x, m1, m2, g};
+    for (int i = 0; i < 4; ++i)
+        for (int j = i + 1; j < 4; ++j)
+            if (overlap(bufs[i], bytes, bufs[j], bytes)) return DPPF_ERR_INVALID_ARG;
+    return DPPF_OK;
+}
+
+int launch_adamw_step(float *x, const AdamArgs &p, int M, int64_t d, int64_t ld, int dev, cudaStream_t s) {
+    const int sms = sm_count(dev);
+    if (sms <= 0) return DPPF_ERR_CUDA;
+    const long long nvec = d / 4;
+    long long bx = (nvec + kThreads - 1) / kThreads;
+    const long long cap = ((long long)sms * 3 + M - 1) / M;
+    if (bx > cap) bx = cap;
+    if (bx < 1) bx = 1;
+    adamw_step_kernel<<<dim3((unsigned)bx, (unsigned)M), kThreads, 0, s>>>(x, p, d, ld, nvec);
+    return cudaGetLastError() == cudaSuccess ? DPPF_OK : DPPF_ERR_CUDA;
+}
+
+template <int M>
+int launch_adamw_round_m(const RoundArgs &a, const AdamArgs &p, int dev, cudaStream_t s) {
+    constexpr int T = Tuning<M>::kThreads;
+    const int sms = sm_count(dev);
+    if (sms <= 0) return DPPF_ERR_CUDA;
+    const long long tile_vecs = (long long)T * Tuning<M>::kUnrollB;
+    long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
+    if (ntiles < 1) ntiles = 1;
+    long long grid = (long long)sms * Tuning<M>::kBlocksPerSM;
+    if (grid > ntiles) grid = ntiles;
+    if (grid > kMaxBlocksSmallM) grid = kMaxBlocksSmallM;
+    adamw_distance_kernel<M><<<(unsigned)grid, T, 0, s>>>(a, p);
+    update_kernel<M, false><<<(unsigned)grid, T, 0, s>>>(a, (int)grid);
+    return cudaGetLastError() == cudaSuccess ? DPPF_OK : DPPF_ERR_CUDA;
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------- C ABI
@@ -1517,6 +1718,59 @@ int dppf_consensus_general(float *x, int M, int64_t d, int64_t ld, float alpha, 
     switch (M) {
 #define DPPF_CASE(MM) case MM: return launch_general_m<MM>(a, dev, s);
         DPPF_CASE(1) DPPF_CASE(2) DPPF_CASE(3) DPPF_CASE(4) DPPF_CASE(5) DPPF_CASE(6) DPPF_CASE(7) DPPF_CASE(8)
+        DPPF_CASE(9) DPPF_CASE(10) DPPF_CASE(11) DPPF_CASE(12) DPPF_CASE(13) DPPF_CASE(14) DPPF_CASE(15)
+        DPPF_CASE(16)
+#undef DPPF_CASE
+        default: return DPPF_ERR_INVALID_ARG;
+    }
+}
+
+int dppf_adamw_step(float *x, float *exp_avg, float *exp_avg_sq, const float *g, int M, int64_t d, int64_t ld,
+                    float lr, float beta1, float beta2, float eps, float weight_decay, int step, void *cuda_stream) {
+    int rc = check_adam_buffers(x, exp_avg, exp_avg_sq, g, M, d, ld);
+    if (rc != DPPF_OK) return rc;
+    AdamArgs p;
+    if ((rc = make_adam_args(exp_avg, exp_avg_sq, g, lr, beta1, beta2, eps, weight_decay, step, &p)) != DPPF_OK) return rc;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DPPF_ERR_CUDA;
+    return launch_adamw_step(x, p, M, d, ld, dev, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int dppf_adamw_step_and_consensus(float *x, float *exp_avg, float *exp_avg_sq, const float *g, int M, int64_t d,
+                                  int64_t ld, float lr, float beta1, float beta2, float eps, float weight_decay,
+                                  int step, float alpha, float lambda, float *norms_out, void *ws, size_t ws_bytes,
+                                  void *cuda_stream) {
+    int rc = check_adam_buffers(x, exp_avg, exp_avg_sq, g, M, d, ld);
+    if (rc != DPPF_OK) return rc;
+    if (M > kMaxTemplateM) return DPPF_ERR_INVALID_ARG;
+    if (!finite_all({alpha, lambda})) return DPPF_ERR_INVALID_ARG;
+    AdamArgs p;
+    if ((rc = make_adam_args(exp_avg, exp_avg_sq, g, lr, beta1, beta2, eps, weight_decay, step, &p)) != DPPF_OK) return rc;
+    if (!ws) return DPPF_ERR_INVALID_ARG;
+    if (!aligned128(ws)) return DPPF_ERR_ALIGNMENT;
+    if (ws_bytes < workspace_bytes(M)) return DPPF_ERR_WORKSPACE;
+    const size_t bytes = (size_t)M * (size_t)ld * sizeof(float);
+    if (overlap(x, bytes, ws, workspace_bytes(M))) return DPPF_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DPPF_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    RoundArgs a;
+    a.x = x; a.v = nullptr; a.g = g;
+    a.d = d; a.ld = ld; a.nvec = d / 4;
+    a.alpha = alpha; a.lambda = lambda; a.lr = 0.f; a.mu = 0.f; a.wd = 0.f;
+    a.norms_out = norms_out;
+    a.hdr = reinterpret_cast<WsHeader *>(ws);
+    a.partials = reinterpret_cast<double *>(static_cast<unsigned char *>(ws) + kHeaderBytes);
+    a.norms_stage = reinterpret_cast<float *>(static_cast<unsigned char *>(ws) + norms_stage_offset(M));
+    a.M = M;
+    if (M == 1) {
+        if ((rc = launch_adamw_step(x, p, M, d, ld, dev, s)) != DPPF_OK) return rc;
+        zero_norms_kernel<<<1, 32, 0, s>>>(norms_out, a.norms_stage, a.hdr);
+        return cudaGetLastError() == cudaSuccess ? DPPF_OK : DPPF_ERR_CUDA;
+    }
+    switch (M) {
+#define DPPF_CASE(MM) case MM: return launch_adamw_round_m<MM>(a, p, dev, s);
+        DPPF_CASE(2) DPPF_CASE(3) DPPF_CASE(4) DPPF_CASE(5) DPPF_CASE(6) DPPF_CASE(7) DPPF_CASE(8)
         DPPF_CASE(9) DPPF_CASE(10) DPPF_CASE(11) DPPF_CASE(12) DPPF_CASE(13) DPPF_CASE(14) DPPF_CASE(15)
         DPPF_CASE(16)
 #undef DPPF_CASE
