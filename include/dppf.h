@@ -201,6 +201,31 @@ int dppf_consensus_static(float *x, int M, int64_t d, int64_t ld, float alpha, f
                           float *norms_out, void *cuda_stream);
 
 /*
+ * Host-side scalars of a DPPF run (no device work, no CUDA call).
+ *
+ * dppf_lambda_schedule: push strength at iteration t of T (appendix, "How to schedule the
+ *   pushing force?"): FIXED lambda; DECREASING lambda/2 (1 + cos(t pi / T)) (follows the
+ *   cosine-annealed learning rate); INCREASING lambda/2 (1 - cos(t pi / T)) (the schedule
+ *   the paper adopts).  NaN for an unknown kind, T <= 0 or t < 0.
+ * dppf_lr_cosine: cosine annealing lr_max/2 (1 + cos(t pi / T)).
+ * dppf_qsr_period: communication period of the quadratic synchronisation rule the paper
+ *   compares with ("Comparison with Other Communication-Efficient Methods"): max(tau_base, floor((beta / lr_t)^2)); -1 on bad arguments.
+ * dppf_round_metrics: from the M pre-round distances r_m (HOST fp32[M], as written to
+ *   norms_out and copied back): their mean (the relaxed Mean Valley measure the ablation
+ *   plots), the pull strength alpha * r_m per worker (host fp32[M] or NULL) and the push
+ *   strength lambda (the push is unit-normed), the two forces whose balance the ablation of
+ *   the pull-push mechanism tracks.  Output pointers may be NULL.
+ */
+#define DPPF_SCHEDULE_FIXED 0
+#define DPPF_SCHEDULE_DECREASING 1
+#define DPPF_SCHEDULE_INCREASING 2
+float dppf_lambda_schedule(int kind, float lambda, int64_t t, int64_t T);
+float dppf_lr_cosine(float lr_max, int64_t t, int64_t T);
+int64_t dppf_qsr_period(int64_t tau_base, float beta, float lr_t);
+int dppf_round_metrics(const float *norms_host, int M, float alpha, float lambda, float *mean_distance,
+                       float *pull_strength, float *push_strength);
+
+/*
  * Synchronises `cuda_stream` and returns the status word the kernels keep in the
  * workspace header: DPPF_OK; DPPF_ERR_WORKSPACE if the update pass found a
  * header that its distance pass did not write (workspace overwritten between the

@@ -21,7 +21,8 @@ EXPORTS = ("dppf_workspace_bytes", "dppf_consensus", "dppf_consensus_ex", "dppf_
            "dppf_local_step_and_consensus", "dppf_local_step_and_consensus_ex",
            "dppf_consensus_host", "dppf_device_status", "dppf_status_string", "dppf_launch_count",
            "dppf_consensus_static", "dppf_consensus_general",
-           "dppf_adamw_step", "dppf_adamw_step_and_consensus")
+           "dppf_adamw_step", "dppf_adamw_step_and_consensus",
+           "dppf_lambda_schedule", "dppf_lr_cosine", "dppf_qsr_period", "dppf_round_metrics")
 
 _lib = None
 
@@ -57,6 +58,15 @@ def load(rebuild_if_stale: bool = False) -> ctypes.CDLL:
     lib.dppf_local_step_and_consensus_ex.argtypes = [vp, vp, vp, i32, i64, i64, f32, f32, f32, f32, f32, vp, vp, sz, i32, vp]
     lib.dppf_consensus_host.argtypes = [vp, i32, i64, i64, f32, f32, vp, vp, vp, sz, vp]
     lib.dppf_device_status.argtypes = [vp, vp]
+    lib.dppf_lambda_schedule.argtypes = [i32, f32, i64, i64]
+    lib.dppf_lambda_schedule.restype = f32
+    lib.dppf_lr_cosine.argtypes = [f32, i64, i64]
+    lib.dppf_lr_cosine.restype = f32
+    lib.dppf_qsr_period.argtypes = [i64, f32, f32]
+    lib.dppf_qsr_period.restype = i64
+    lib.dppf_round_metrics.argtypes = [ctypes.POINTER(f32), i32, f32, f32, ctypes.POINTER(f32),
+                                       ctypes.POINTER(f32), ctypes.POINTER(f32)]
+    lib.dppf_round_metrics.restype = i32
     lib.dppf_adamw_step.argtypes = [vp, vp, vp, vp, i32, i64, i64, f32, f32, f32, f32, f32, i32, vp]
     lib.dppf_adamw_step.restype = i32
     lib.dppf_adamw_step_and_consensus.argtypes = [vp, vp, vp, vp, i32, i64, i64, f32, f32, f32, f32, f32, i32,
@@ -218,6 +228,32 @@ def dppf_consensus_host(x_host, alpha, lam, norms_host, x_dev, ws, d=None):
     rc = load().dppf_consensus_host(x_host.data_ptr(), M, d, ld, alpha, lam, _ptr(norms_host),
                                     x_dev.data_ptr(), ws.data_ptr(), ws.numel(), _stream())
     _check(rc, "dppf_consensus_host")
+
+
+SCHEDULE_FIXED, SCHEDULE_DECREASING, SCHEDULE_INCREASING = 0, 1, 2
+
+
+def dppf_lambda_schedule(kind, lam, t, T) -> float:
+    return float(load().dppf_lambda_schedule(int(kind), lam, int(t), int(T)))
+
+
+def dppf_lr_cosine(lr_max, t, T) -> float:
+    return float(load().dppf_lr_cosine(lr_max, int(t), int(T)))
+
+
+def dppf_qsr_period(tau_base, beta, lr_t) -> int:
+    return int(load().dppf_qsr_period(int(tau_base), beta, lr_t))
+
+
+def dppf_round_metrics(norms, alpha, lam):
+    """(mean distance, [pull strength per worker], push strength) from host distances."""
+    M = len(norms)
+    arr = (ctypes.c_float * M)(*[float(v) for v in norms])
+    pull = (ctypes.c_float * M)()
+    mean, push = ctypes.c_float(), ctypes.c_float()
+    _check(load().dppf_round_metrics(arr, M, alpha, lam, ctypes.byref(mean), pull, ctypes.byref(push)),
+           "dppf_round_metrics")
+    return mean.value, list(pull), push.value
 
 
 def dppf_device_status(ws) -> int:

@@ -26,6 +26,7 @@
 #include <cuda_runtime.h>
 
 #include <atomic>
+#include <climits>
 #include <cmath>
 #include <cstdint>
 
@@ -1776,6 +1777,45 @@ int dppf_adamw_step_and_consensus(float *x, float *exp_avg, float *exp_avg_sq, c
 #undef DPPF_CASE
         default: return DPPF_ERR_INVALID_ARG;
     }
+}
+
+// ---- host-side scalars of a run (no device work)
+
+float dppf_lambda_schedule(int kind, float lambda, int64_t t, int64_t T) {
+    if (kind == DPPF_SCHEDULE_FIXED) return lambda;
+    if (T <= 0 || t < 0 || (kind != DPPF_SCHEDULE_DECREASING && kind != DPPF_SCHEDULE_INCREASING))
+        return std::nanf("");
+    const double c = std::cos(3.14159265358979323846 * (double)t / (double)T);
+    const double f = (kind == DPPF_SCHEDULE_DECREASING) ? 0.5 * (1.0 + c) : 0.5 * (1.0 - c);
+    return (float)((double)lambda * f);
+}
+
+float dppf_lr_cosine(float lr_max, int64_t t, int64_t T) {
+    if (T <= 0 || t < 0) return std::nanf("");
+    return (float)((double)lr_max * 0.5 * (1.0 + std::cos(3.14159265358979323846 * (double)t / (double)T)));
+}
+
+int64_t dppf_qsr_period(int64_t tau_base, float beta, float lr_t) {
+    if (tau_base < 1 || !std::isfinite(beta) || !std::isfinite(lr_t) || !(lr_t > 0.f)) return -1;
+    const double q = (double)beta / (double)lr_t;
+    const double sq = std::floor(q * q);
+    if (!(sq < 9.0e18)) return INT64_MAX;
+    const int64_t tau = (int64_t)sq;
+    return tau > tau_base ? tau : tau_base;
+}
+
+int dppf_round_metrics(const float *norms_host, int M, float alpha, float lambda, float *mean_distance,
+                       float *pull_strength, float *push_strength) {
+    if (!norms_host || M < 1 || !finite_all({alpha, lambda})) return DPPF_ERR_INVALID_ARG;
+    double sum = 0.0;
+    for (int m = 0; m < M; ++m) {
+        if (!(norms_host[m] >= 0.f)) return DPPF_ERR_INVALID_ARG;
+        sum += (double)norms_host[m];
+        if (pull_strength) pull_strength[m] = (float)((double)alpha * (double)norms_host[m]);
+    }
+    if (mean_distance) *mean_distance = (float)(sum / (double)M);
+    if (push_strength) *push_strength = lambda;
+    return DPPF_OK;
 }
 
 }  // extern "C"

@@ -126,6 +126,29 @@ def test_norms_out_is_optional_and_iterated_rounds_follow_oracle(oracle):
     assert_parity(x.cpu().numpy(), norms.cpu().numpy(), ref, r_ref, d)
 
 
+def test_scheduled_rounds_follow_oracle_and_metrics():
+    """Thirty rounds with the increasing push schedule; distances copied back each round feed
+    the metric helper (mean distance, pull vs push strength)."""
+    import torch
+    import oracle
+    oracle.build()
+    _, binding = require_gpu()
+    d, M, T, alpha, lam = 300_001, 4, 30, 0.1, 0.05
+    x_np = random_replicas(M, d, seed=29)
+    x = to_dev(x_np)
+    ws = binding.alloc_workspace(M, d)
+    norms = torch.zeros(M, device="cuda")
+    ref = x_np
+    for t in range(1, T + 1):
+        lam_t = binding.dppf_lambda_schedule(binding.SCHEDULE_INCREASING, lam, t, T)
+        binding.dppf_consensus(x, alpha, lam_t, norms_out=norms, ws=ws, d=d)
+        ref, r_ref = oracle.consensus(ref, alpha, lam_t, d=d)
+        mean, pull, push = binding.dppf_round_metrics(norms.cpu().tolist(), alpha, lam_t)
+        assert abs(mean - r_ref.mean()) <= 1e-5 * r_ref.mean() and push == pytest.approx(lam_t)
+        np.testing.assert_allclose(pull, np.float32(alpha) * r_ref, rtol=2e-5)
+    assert_parity(x.cpu().numpy(), norms.cpu().numpy(), ref, r_ref, d)
+
+
 @pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("M,d,tau", [(4, 1_000_003, 8), (2, 33, 3), (8, 200_001, 2), (16, 50_001, 2), (18, 40_003, 2), (1, 1000, 2)])
 def test_local_steps_then_fused_round(oracle, M, d, tau, path):
