@@ -1,4 +1,11 @@
-// DPPF consensus round for one B200 (sm_100a): kernels and the C ABI of include/dppf.h.
+// DPPF consensus round for one B200 (sm_100a): host side and the C ABI of include/dppf.h.
+// Kernels live in the .cuh files included below (one translation unit):
+//   common.cuh          constants, argument structs, cache-hinted accesses, rounded arithmetic
+//   round_register.cuh  register-resident round kernels (two-launch and cooperative schedules)
+//   adamw.cuh           AdamW local step, stand-alone and fused into the distance pass
+//   round_staged.cuh    staged persistent round kernel (bulk async copies into a shared-memory ring)
+//   round_general.cuh   general round (weighted consensus variable, push reference, two-term push)
+//   round_generic.cuh   any worker count up to 1024, stand-alone SGD-momentum local step
 //
 // Data layout: x[M, ld] fp32, one row per worker, rows 128-byte aligned.  A "vector" is
 // one float4 (four consecutive columns of one row); a thread always handles the same
@@ -22,1188 +29,14 @@
 // makes the zero-distance round leave x bit-for-bit unchanged.
 #include "dppf.h"
 
-#include <cooperative_groups.h>
-#include <cuda_runtime.h>
-
-#include <atomic>
-#include <climits>
-#include <cmath>
-#include <cstdint>
-
-namespace cg = cooperative_groups;
+#include "common.cuh"
+#include "round_register.cuh"
+#include "adamw.cuh"
+#include "round_staged.cuh"
+#include "round_general.cuh"
+#include "round_generic.cuh"
 
 namespace {
-
-constexpr int kThreads = 256;            // threads per block: generic and local-step kernels
-constexpr int kWarps = kThreads / 32;
-constexpr int kMaxTemplateM = 16;        // worker counts with register-resident kernels
-constexpr int kMaxBlocksSmallM = 2048;   // partial-sum slots reserved per worker, M <= 16
-constexpr int kMaxBlocksLargeM = 512;    // ... and for the generic kernels
-constexpr size_t kHeaderBytes = 256;
-constexpr unsigned kMagic = 0x44505046u; // "DPPF"
-
-struct WsHeader {
-    int status;       // dppf_status seen by the kernels
-    unsigned magic;   // written by the distance pass, checked by the update pass
-    int grid;         // blocks that wrote partials
-    int M;
-};
-
-struct RoundArgs {
-    float *x;
-    float *v;         // fused local step only
-    const float *g;   // fused local step only
-    long long d, ld, nvec;   // nvec = d / 4 full float4 groups per row
-    float alpha, lambda, lr, mu, wd;
-    float *norms_out; // may be null
-    float *norms_stage; // fp32[M] inside the workspace (always written)
-    WsHeader *hdr;
-    double *partials; // [grid, M]
-    int M;            // runtime copy (generic kernels)
-};
-
-// ---------------------------------------------------------------- memory access helpers
-
-__device__ __forceinline__ float4 ld_keep(const float *p) {   // normal L2 priority, skip L1
-    return __ldcg(reinterpret_cast<const float4 *>(p));
-}
-__device__ __forceinline__ float4 ld_last_use(const float *p) {  // evict-first: dead after this read
-    return __ldcs(reinterpret_cast<const float4 *>(p));
-}
-__device__ __forceinline__ void st_keep(float *p, float4 v) {
-    __stcg(reinterpret_cast<float4 *>(p), v);
-}
-
-// ---------------------------------------------------------------- arithmetic helpers
-// Explicitly rounded operations: the compiler may not re-associate or contract them, so
-// the distance pass and the update pass see bit-identical deviations.
-
-__device__ __forceinline__ float4 sub4(float4 a, float4 b) {
-    return make_float4(__fsub_rn(a.x, b.x), __fsub_rn(a.y, b.y), __fsub_rn(a.z, b.z), __fsub_rn(a.w, b.w));
-}
-__device__ __forceinline__ float4 add4(float4 a, float4 b) {
-    return make_float4(__fadd_rn(a.x, b.x), __fadd_rn(a.y, b.y), __fadd_rn(a.z, b.z), __fadd_rn(a.w, b.w));
-}
-__device__ __forceinline__ float4 scale4(float4 a, float s) {
-    return make_float4(__fmul_rn(a.x, s), __fmul_rn(a.y, s), __fmul_rn(a.z, s), __fmul_rn(a.w, s));
-}
-__device__ __forceinline__ float sq_acc(float acc, float4 d) {
-    acc = __fmaf_rn(d.x, d.x, acc);
-    acc = __fmaf_rn(d.y, d.y, acc);
-    acc = __fmaf_rn(d.z, d.z, acc);
-    acc = __fmaf_rn(d.w, d.w, acc);
-    return acc;
-}
-// x - c * dev
-__device__ __forceinline__ float4 apply4(float4 x, float4 dev, float c) {
-    return make_float4(__fmaf_rn(-c, dev.x, x.x), __fmaf_rn(-c, dev.y, x.y),
-                       __fmaf_rn(-c, dev.z, x.z), __fmaf_rn(-c, dev.w, x.w));
-}
-// Local optimiser step on one element: g~ = g + wd x ; v' = mu v + g~ ; x' = x - lr v'.
-__device__ __forceinline__ void sgd1(float &x, float &v, float g, float lr, float mu, float wd) {
-    float gt = __fmaf_rn(wd, x, g);
-    v = __fmaf_rn(mu, v, gt);
-    x = __fmaf_rn(-lr, v, x);
-}
-__device__ __forceinline__ void sgd4(float4 &x, float4 &v, float4 g, float lr, float mu, float wd) {
-    sgd1(x.x, v.x, g.x, lr, mu, wd);
-    sgd1(x.y, v.y, g.y, lr, mu, wd);
-    sgd1(x.z, v.z, g.z, lr, mu, wd);
-    sgd1(x.w, v.w, g.w, lr, mu, wd);
-}
-
-// Shifted mean of one vector over the M rows: ebar = (sum_{m>=1} (x_m - x_0)) / M, so that
-// x_A = x_0 + ebar and the deviation of row m is dev_m = (x_m - x_0) - ebar (dev_0 = -ebar).
-template <int M>
-__device__ __forceinline__ float4 shifted_mean(const float4 (&xv)[M]) {
-    const float inv_m = 1.0f / (float)M;
-    float4 esum = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-    for (int m = 1; m < M; ++m) esum = add4(esum, sub4(xv[m], xv[0]));
-    return scale4(esum, inv_m);
-}
-__device__ __forceinline__ float4 deviation(float4 xm, float4 x0, float4 ebar, int m) {
-    if (m == 0) return make_float4(-ebar.x, -ebar.y, -ebar.z, -ebar.w);
-    return sub4(sub4(xm, x0), ebar);
-}
-
-__device__ __forceinline__ double warp_sum(double a) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-    return a;   // butterfly: every lane holds the same bits
-}
-
-// Coefficient c_m = alpha - lambda / r_m of the single-line update.  Zero distance: the push
-// direction is undefined and the pull acts on a zero vector, so the replica must stay as it
-// is, bit for bit (including the sign of zeros).  That case is signalled by a NaN coefficient,
-// which the update pass reads as "do not write this row".
-__device__ __forceinline__ float coefficient(double S, float alpha, float lambda, float *r_out) {
-    double r = sqrt(S);
-    *r_out = (float)r;
-    if (!(r > 0.0)) return __int_as_float(0x7fc00000);
-    return (float)((double)alpha - (double)lambda / r);
-}
-__device__ __forceinline__ bool row_is_written(float c) { return c == c; }
-
-// ---------------------------------------------------------------- register-resident kernels (M <= 16)
-
-// Launch shape per worker count, from sweeps on B200.  The update pass mixes reads and
-// writes and is fastest with about 40-48 KB of loads in flight per SM; more outstanding
-// requests lower its DRAM efficiency, fewer cannot cover the latency.  The read-only distance
-// pass wants about twice that, which it gets from a deeper unroll on the same grid.
-//   bytes in flight per SM = kThreads * kBlocksPerSM * unroll * M * 16
-template <int M>
-struct Tuning {
-    static constexpr int kThreads =
-        (M <= 2) ? 320 : (M == 3) ? 384 : (M == 4) ? 320 : (M == 5) ? 288 : (M == 6) ? 224 :
-        (M <= 8) ? 192 : (M == 9) ? 320 : (M == 10) ? 288 : (M <= 12) ? 256 : 224;
-    static constexpr int kBlocksPerSM = (M <= 8) ? 2 : 1;
-    static constexpr int kUnrollA = (M <= 2) ? 4 : (M <= 8) ? 2 : 1;      // distance pass
-    static constexpr int kUnrollB = (M <= 2) ? 2 : 1;                     // update pass
-    // With the local step fused in, the distance pass moves five streams per row (x, v, g in,
-    // x, v out) and peaks at about half the resident threads (~60 KB of loads in flight per
-    // SM); the update pass of that launch doubles its unroll to keep its own 40-48 KB.
-    static constexpr int kBlocksPerSMFused = (kBlocksPerSM > 1) ? kBlocksPerSM / 2 : 1;
-    static constexpr int kUnrollFused = 1;
-    static constexpr int kUnrollBFused = kUnrollB * (kBlocksPerSM / kBlocksPerSMFused);
-    static constexpr int kWarps = kThreads / 32;
-
-};
-
-// Scalar tail: columns 4*nvec .. d-1 (at most three), handled by one thread of block 0.
-template <int M, bool kLocalStep>
-__device__ __forceinline__ void tail_distance(const RoundArgs &a, float (&acc)[M]) {
-    const float inv_m = 1.0f / (float)M;
-    for (long long i = a.nvec * 4; i < a.d; ++i) {
-        float xs[M];
-#pragma unroll
-        for (int m = 0; m < M; ++m) {
-            float xi = a.x[m * a.ld + i];
-            if (kLocalStep) {
-                float vi = a.v[m * a.ld + i];
-                sgd1(xi, vi, a.g[m * a.ld + i], a.lr, a.mu, a.wd);
-                a.v[m * a.ld + i] = vi;
-                a.x[m * a.ld + i] = xi;
-            }
-            xs[m] = xi;
-        }
-        float esum = 0.f;
-#pragma unroll
-        for (int m = 1; m < M; ++m) { xs[m] = __fsub_rn(xs[m], xs[0]); esum = __fadd_rn(esum, xs[m]); }
-        const float ebar = __fmul_rn(esum, inv_m);
-        acc[0] = __fmaf_rn(ebar, ebar, acc[0]);
-#pragma unroll
-        for (int m = 1; m < M; ++m) { float dv = __fsub_rn(xs[m], ebar); acc[m] = __fmaf_rn(dv, dv, acc[m]); }
-    }
-}
-
-template <int M>
-__device__ __forceinline__ void tail_update(const RoundArgs &a, const float *c) {
-    const float inv_m = 1.0f / (float)M;
-    for (long long i = a.nvec * 4; i < a.d; ++i) {
-        float xs[M], dv[M];
-#pragma unroll
-        for (int m = 0; m < M; ++m) xs[m] = a.x[m * a.ld + i];
-        float esum = 0.f;
-#pragma unroll
-        for (int m = 1; m < M; ++m) { dv[m] = __fsub_rn(xs[m], xs[0]); esum = __fadd_rn(esum, dv[m]); }
-        const float ebar = __fmul_rn(esum, inv_m);
-        dv[0] = -ebar;
-#pragma unroll
-        for (int m = 1; m < M; ++m) dv[m] = __fsub_rn(dv[m], ebar);
-#pragma unroll
-        for (int m = 0; m < M; ++m)
-            if (row_is_written(c[m])) a.x[m * a.ld + i] = __fmaf_rn(-c[m], dv[m], xs[m]);
-    }
-}
-
-// Distance pass body.  Tile t of the block = vectors [(t*U+u)*T + tid], u < U.
-template <int M, bool kLocalStep>
-__device__ __forceinline__ void distance_pass(const RoundArgs &a, double *s_red /* [warps][M] */) {
-    constexpr int U = kLocalStep ? Tuning<M>::kUnrollFused : Tuning<M>::kUnrollA;
-    constexpr int T = Tuning<M>::kThreads;
-    const long long tile_vecs = (long long)T * U;
-    const long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
-    float acc[M];
-#pragma unroll
-    for (int m = 0; m < M; ++m) acc[m] = 0.f;
-
-    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
-        float4 xv[U][M];
-        bool live[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const long long j = (t * U + u) * T + threadIdx.x;
-            live[u] = j < a.nvec;
-            if (live[u]) {
-                if (kLocalStep) {
-                    // Rows in groups of four: all loads of a group are issued before its first
-                    // store (x, v, g may not alias, but the compiler cannot know that and
-                    // would otherwise order every row's loads behind the previous row's stores).
-                    constexpr int G = 4;
-#pragma unroll
-                    for (int m0 = 0; m0 < M; m0 += G) {
-                        float4 vv[G], gv[G];
-#pragma unroll
-                        for (int k = 0; k < G; ++k) {
-                            if (m0 + k < M) {
-                                const long long off = (m0 + k) * a.ld + j * 4;
-                                xv[u][m0 + k] = ld_last_use(a.x + off);
-                                vv[k] = ld_last_use(a.v + off);
-                                gv[k] = ld_last_use(a.g + off);
-                            }
-                        }
-#pragma unroll
-                        for (int k = 0; k < G; ++k) {
-                            if (m0 + k < M) {
-                                const long long off = (m0 + k) * a.ld + j * 4;
-                                sgd4(xv[u][m0 + k], vv[k], gv[k], a.lr, a.mu, a.wd);
-                                st_keep(a.v + off, vv[k]);
-                                st_keep(a.x + off, xv[u][m0 + k]);
-                            }
-                        }
-                    }
-                } else {
-#pragma unroll
-                    for (int m = 0; m < M; ++m) xv[u][m] = ld_keep(a.x + m * a.ld + j * 4);
-                }
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (live[u]) {
-                const float4 ebar = shifted_mean<M>(xv[u]);
-#pragma unroll
-                for (int m = 0; m < M; ++m) acc[m] = sq_acc(acc[m], deviation(xv[u][m], xv[u][0], ebar, m));
-            }
-        }
-    }
-    if (blockIdx.x == 0 && threadIdx.x == 0) tail_distance<M, kLocalStep>(a, acc);
-
-    // thread -> warp (butterfly, fp64) -> block (warp order) -> one fp64 partial per worker
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int m = 0; m < M; ++m) {
-        double s = warp_sum((double)acc[m]);
-        if (lane == 0) s_red[warp * M + m] = s;
-    }
-    __syncthreads();
-    if (threadIdx.x < M) {
-        double s = 0.0;
-        for (int w = 0; w < Tuning<M>::kWarps; ++w) s += s_red[w * M + threadIdx.x];
-        a.partials[(long long)blockIdx.x * M + threadIdx.x] = s;
-    }
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        a.hdr->status = DPPF_OK;
-        a.hdr->magic = kMagic;
-        a.hdr->grid = (int)gridDim.x;
-        a.hdr->M = M;
-    }
-}
-
-// Cross-block sum in block order, identical in every block; fills s_c[M] and reports r_m.
-// Returns false if the workspace header does not describe this launch.
-__device__ __forceinline__ bool finalise(const RoundArgs &a, int M, int nblocks, float *s_c, int *s_ok) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0)
-        *s_ok = (a.hdr->magic == kMagic && a.hdr->grid == nblocks && a.hdr->M == M) ? 1 : 0;
-    const int nwarps = blockDim.x >> 5;
-    for (int m = warp; m < M; m += nwarps) {
-        double s = 0.0;
-        for (int b = lane; b < nblocks; b += 32) s += __ldcg(a.partials + (long long)b * M + m);
-        s = warp_sum(s);
-        if (lane == 0) {
-            float r;
-            s_c[m] = coefficient(s, a.alpha, a.lambda, &r);
-            if (blockIdx.x == 0) {
-                a.norms_stage[m] = r;
-                if (a.norms_out) a.norms_out[m] = r;
-            }
-        }
-    }
-    __syncthreads();
-    if (!*s_ok && blockIdx.x == 0 && threadIdx.x == 0) a.hdr->status = DPPF_ERR_WORKSPACE;
-    return *s_ok != 0;
-}
-
-template <int M, int U>
-__device__ __forceinline__ void update_pass(const RoundArgs &a, const float *s_c) {
-    constexpr int T = Tuning<M>::kThreads;
-    const long long tile_vecs = (long long)T * U;
-    const long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
-    const float *c = s_c;
-    if (ntiles > blockIdx.x) {
-        // last tile of this block's static sequence, then backwards
-        long long t = blockIdx.x + (ntiles - 1 - blockIdx.x) / gridDim.x * gridDim.x;
-        for (; t >= 0; t -= gridDim.x) {
-            float4 xv[U][M];
-            bool live[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const long long j = (t * U + u) * T + threadIdx.x;
-                live[u] = j < a.nvec;
-                if (live[u]) {
-#pragma unroll
-                    for (int m = 0; m < M; ++m) xv[u][m] = ld_last_use(a.x + m * a.ld + j * 4);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                if (live[u]) {
-                    const long long j = (t * U + u) * T + threadIdx.x;
-                    const float4 ebar = shifted_mean<M>(xv[u]);
-#pragma unroll
-                    for (int m = 0; m < M; ++m)
-                        if (row_is_written(c[m]))
-                            st_keep(a.x + m * a.ld + j * 4,
-                                    apply4(xv[u][m], deviation(xv[u][m], xv[u][0], ebar, m), c[m]));
-                }
-            }
-        }
-    }
-    if (blockIdx.x == 0 && threadIdx.x == 0) tail_update<M>(a, c);
-}
-
-template <int M, bool kLocalStep>
-__global__ void __launch_bounds__(Tuning<M>::kThreads, (kLocalStep ? Tuning<M>::kBlocksPerSMFused : Tuning<M>::kBlocksPerSM))
-distance_kernel(const RoundArgs a) {
-    __shared__ double s_red[Tuning<M>::kWarps * M];
-    distance_pass<M, kLocalStep>(a, s_red);
-}
-
-template <int M, bool kAfterLocalStep>
-__global__ void __launch_bounds__(Tuning<M>::kThreads, (kAfterLocalStep ? Tuning<M>::kBlocksPerSMFused : Tuning<M>::kBlocksPerSM))
-update_kernel(const RoundArgs a, int nblocks_a) {
-    __shared__ float s_c[M];
-    __shared__ int s_ok;
-    if (!finalise(a, M, nblocks_a, s_c, &s_ok)) return;
-    update_pass<M, (kAfterLocalStep ? Tuning<M>::kUnrollBFused : Tuning<M>::kUnrollB)>(a, s_c);
-}
-
-// One persistent launch: distance pass, grid-wide barrier, update pass.  Launched with
-// cudaLaunchCooperativeKernel, which refuses the launch unless all blocks are co-resident.
-template <int M, bool kLocalStep>
-__global__ void __launch_bounds__(Tuning<M>::kThreads, (kLocalStep ? Tuning<M>::kBlocksPerSMFused : Tuning<M>::kBlocksPerSM))
-round_kernel(const RoundArgs a) {
-    __shared__ double s_red[Tuning<M>::kWarps * M];
-    __shared__ float s_c[M];
-    __shared__ int s_ok;
-    distance_pass<M, kLocalStep>(a, s_red);
-    cg::this_grid().sync();
-    if (!finalise(a, M, (int)gridDim.x, s_c, &s_ok)) return;
-    update_pass<M, (kLocalStep ? Tuning<M>::kUnrollBFused : Tuning<M>::kUnrollB)>(a, s_c);
-}
-
-// ---------------------------------------------------------------- AdamW local step (fused and stand-alone)
-// The ViT runs of the paper train with AdamW (lr 5e-4, weight decay 0.01).  Decoupled form:
-//   x <- x (1 - lr wd);  m <- m + (1 - b1)(g - m);  v <- b2 v + (1 - b2) g^2;
-//   x <- x - [lr / (1 - b1^t)] m / ( sqrt(v) / sqrt(1 - b2^t) + eps )
-// The step-dependent factors are formed on the host in double and passed as floats.
-
-struct AdamArgs {
-    float *m1;   // exp_avg      [M, ld]
-    float *m2;   // exp_avg_sq   [M, ld]
-    const float *g;
-    float decay, one_minus_b1, b2, one_minus_b2, step_size, inv_sqrt_bc2, eps;
-};
-
-__device__ __forceinline__ void adamw1(float &x, float &m1, float &m2, float g, const AdamArgs &p) {
-    x = __fmul_rn(x, p.decay);
-    m1 = __fmaf_rn(p.one_minus_b1, __fsub_rn(g, m1), m1);
-    m2 = __fmaf_rn(p.b2, m2, __fmul_rn(p.one_minus_b2, __fmul_rn(g, g)));
-    const float denom = __fmaf_rn(__fsqrt_rn(m2), p.inv_sqrt_bc2, p.eps);
-    x = __fmaf_rn(-p.step_size, __fdiv_rn(m1, denom), x);
-}
-__device__ __forceinline__ void adamw4(float4 &x, float4 &m1, float4 &m2, float4 g, const AdamArgs &p) {
-    adamw1(x.x, m1.x, m2.x, g.x, p);
-    adamw1(x.y, m1.y, m2.y, g.y, p);
-    adamw1(x.z, m1.z, m2.z, g.z, p);
-    adamw1(x.w, m1.w, m2.w, g.w, p);
-}
-
-// Distance pass with the AdamW step applied first; leaves the same partial sums and header
-// as distance_kernel, so update_kernel<M, false> completes the round.  Measured best with
-// the plain round's residency and two rows of loads in flight per thread.
-template <int M>
-__global__ void __launch_bounds__(Tuning<M>::kThreads, Tuning<M>::kBlocksPerSM)
-adamw_distance_kernel(const RoundArgs a, const AdamArgs p) {
-    constexpr int T = Tuning<M>::kThreads;
-    constexpr int G = 2;                               // rows whose loads are issued together
-    __shared__ double s_red[Tuning<M>::kWarps * M];
-    const long long ntiles = (a.nvec + T - 1) / T;
-    float acc[M];
-#pragma unroll
-    for (int m = 0; m < M; ++m) acc[m] = 0.f;
-    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
-        const long long j = t * T + threadIdx.x;
-        if (j < a.nvec) {
-            float4 xv[M];
-#pragma unroll
-            for (int m0 = 0; m0 < M; m0 += G) {
-                float4 av[G], bv[G], gv[G];
-#pragma unroll
-                for (int k = 0; k < G; ++k) {
-                    if (m0 + k < M) {
-                        const long long off = (m0 + k) * a.ld + j * 4;
-                        xv[m0 + k] = ld_last_use(a.x + off);
-                        av[k] = ld_last_use(p.m1 + off);
-                        bv[k] = ld_last_use(p.m2 + off);
-                        gv[k] = ld_last_use(p.g + off);
-                    }
-                }
-#pragma unroll
-                for (int k = 0; k < G; ++k) {
-                    if (m0 + k < M) {
-                        const long long off = (m0 + k) * a.ld + j * 4;
-                        adamw4(xv[m0 + k], av[k], bv[k], gv[k], p);
-                        st_keep(p.m1 + off, av[k]);
-                        st_keep(p.m2 + off, bv[k]);
-                        st_keep(a.x + off, xv[m0 + k]);
-                    }
-                }
-            }
-            const float4 ebar = shifted_mean<M>(xv);
-#pragma unroll
-            for (int m = 0; m < M; ++m) acc[m] = sq_acc(acc[m], deviation(xv[m], xv[0], ebar, m));
-        }
-    }
-    if (blockIdx.x == 0 && threadIdx.x == 0) {          // scalar tail columns
-        const float inv_m = 1.0f / (float)M;
-        for (long long i = a.nvec * 4; i < a.d; ++i) {
-            float xs[M];
-#pragma unroll
-            for (int m = 0; m < M; ++m) {
-                const long long off = m * a.ld + i;
-                float xi = a.x[off], ai = p.m1[off], bi = p.m2[off];
-                adamw1(xi, ai, bi, p.g[off], p);
-                p.m1[off] = ai;
-                p.m2[off] = bi;
-                a.x[off] = xi;
-                xs[m] = xi;
-            }
-            float esum = 0.f;
-#pragma unroll
-            for (int m = 1; m < M; ++m) { xs[m] = __fsub_rn(xs[m], xs[0]); esum = __fadd_rn(esum, xs[m]); }
-            const float ebar = __fmul_rn(esum, inv_m);
-            acc[0] = __fmaf_rn(ebar, ebar, acc[0]);
-#pragma unroll
-            for (int m = 1; m < M; ++m) { float dv = __fsub_rn(xs[m], ebar); acc[m] = __fmaf_rn(dv, dv, acc[m]); }
-        }
-    }
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int m = 0; m < M; ++m) {
-        double sum = warp_sum((double)acc[m]);
-        if (lane == 0) s_red[warp * M + m] = sum;
-    }
-    __syncthreads();
-    if (threadIdx.x < M) {
-        double sum = 0.0;
-        for (int w = 0; w < Tuning<M>::kWarps; ++w) sum += s_red[w * M + threadIdx.x];
-        a.partials[(long long)blockIdx.x * M + threadIdx.x] = sum;
-    }
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        a.hdr->status = DPPF_OK;
-        a.hdr->magic = kMagic;
-        a.hdr->grid = (int)gridDim.x;
-        a.hdr->M = M;
-    }
-}
-
-__global__ void __launch_bounds__(kThreads) adamw_step_kernel(float *x, const AdamArgs p, long long d, long long ld,
-                                                              long long nvec) {
-    const long long row = (long long)blockIdx.y * ld;
-    for (long long j = (long long)blockIdx.x * kThreads + threadIdx.x; j < nvec; j += (long long)gridDim.x * kThreads) {
-        const long long off = row + j * 4;
-        float4 xx = ld_last_use(x + off), aa = ld_last_use(p.m1 + off), bb = ld_last_use(p.m2 + off),
-               gg = ld_last_use(p.g + off);
-        adamw4(xx, aa, bb, gg, p);
-        st_keep(p.m1 + off, aa);
-        st_keep(p.m2 + off, bb);
-        st_keep(x + off, xx);
-    }
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        for (long long i = nvec * 4; i < d; ++i) {
-            const long long off = row + i;
-            float xi = x[off], ai = p.m1[off], bi = p.m2[off];
-            adamw1(xi, ai, bi, p.g[off], p);
-            p.m1[off] = ai;
-            p.m2[off] = bi;
-            x[off] = xi;
-        }
-    }
-}
-
-// ---------------------------------------------------------------- staged persistent kernel (default, M <= 16)
-// One block per SM keeps a ring of up to kMaxStages shared-memory stages; a stage holds the same
-// column chunk of all M rows (about 32 KB).  One thread fills stages with 1-D bulk async
-// copies (cp.async.bulk, completion on an mbarrier); all threads then read the chunk from
-// shared memory.  Both passes run in this one cooperative launch:
-//   distance pass  chunks in ascending order, up to kPrefetchA chunks (~96 KB) in flight;
-//   update pass    the same chunks in descending order with one chunk (~32 KB) in flight --
-//                  the read/write mix is fastest with few outstanding loads -- results go
-//                  straight from registers to global memory.
-// The last kStages chunks of the distance pass are still in the ring when the update pass
-// starts, so it consumes them without touching DRAM or L2 again.
-// Every wait on an mbarrier is bounded; if one gives up the block marks its partial sums
-// with a negative value, every block then sees the mark after the grid barrier, nobody
-// writes x, and the status word reports DPPF_ERR_TIMEOUT.
-
-constexpr int kStagedThreads = 256;
-constexpr int kStagedWarps = kStagedThreads / 32;
-constexpr int kMaxStages = 6;
-constexpr int kPrefetchA = 3;
-constexpr int kPrefetchB = 1;
-constexpr int kSpinLimit = 1 << 22;   // mbarrier try_wait polls before a wait gives up (~ a second)
-
-template <int M>
-struct StagedShape {
-    // columns per stage and row: a stage of about 32 KB (40 KB measured best for M = 8)
-    static constexpr int kChunk = (M == 8) ? 1280 : ((8192 / M) / 128) * 128;
-    static constexpr size_t kStageFloats = (size_t)M * kChunk;
-    static constexpr int kFit = (int)((200 * 1024) / (kStageFloats * sizeof(float)));
-    static constexpr int kStages = kFit < kMaxStages ? kFit : kMaxStages;
-    static constexpr size_t kSmemBytes = (size_t)kStages * kStageFloats * sizeof(float);
-    static_assert(kStages > kPrefetchA, "ring must be deeper than the prefetch distance");
-};
-
-__device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(unsigned long long *bar, int count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned long long *bar, unsigned parity) {
-    unsigned ok;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: false if the phase did not complete within kSpinLimit polls.
-__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long *bar, unsigned parity) {
-    for (int spins = 0; spins < kSpinLimit; ++spins)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-// global -> shared bulk copy; dst, src 16-byte aligned, bytes a multiple of 16.
-__device__ __forceinline__ void bulk_load(void *dst_smem, const void *src, unsigned bytes, unsigned long long *bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_addr(dst_smem)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
-}
-
-template <int M>
-__global__ void __launch_bounds__(kStagedThreads, 1) round_kernel_staged(const RoundArgs a) {
-    constexpr int CH = StagedShape<M>::kChunk;
-    constexpr int kStages = StagedShape<M>::kStages;
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    float *ring = reinterpret_cast<float *>(smem_raw);             // [kStages][M][CH]
-    __shared__ unsigned long long full[kStages];
-    __shared__ double s_red[kStagedWarps * M];
-    __shared__ float s_c[M];
-    __shared__ int s_ok;
-    const int tid = threadIdx.x;
-    if (tid == 0) {
-        for (int st = 0; st < kStages; ++st) mbar_init(&full[st], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-
-    const long long d4 = a.nvec * 4;                                // columns covered by float4 groups
-    const long long nchunks = (d4 + CH - 1) / CH;
-    // this block's chunks, by local index k: chunk blockIdx.x + k * gridDim.x, ring stage k % kStages
-    const long long n = (nchunks > blockIdx.x) ? (nchunks - 1 - blockIdx.x) / gridDim.x + 1 : 0;
-    unsigned phase = 0;                                             // bit st: parity of the next wait on stage st
-    int failed = 0;
-
-    auto chunk_cols = [&](long long k) -> int {
-        const long long c0 = (blockIdx.x + k * gridDim.x) * CH;
-        return (int)((d4 - c0 < CH) ? (d4 - c0) : CH);
-    };
-    auto issue = [&](long long k) {                                 // one thread: M row copies into one stage
-        const int st = (int)(k % kStages);
-        const long long c0 = (blockIdx.x + k * gridDim.x) * CH;
-        const unsigned bytes = (unsigned)chunk_cols(k) * 4u;
-        mbar_expect_tx(&full[st], bytes * M);
-#pragma unroll
-        for (int m = 0; m < M; ++m)
-            bulk_load(ring + ((size_t)st * M + m) * CH, a.x + m * a.ld + c0, bytes, &full[st]);
-    };
-
-    // ---- distance pass
-    double acc[M];
-#pragma unroll
-    for (int m = 0; m < M; ++m) acc[m] = 0.0;
-    if (tid == 0)
-        for (long long k = 0; k < kPrefetchA && k < n; ++k) issue(k);
-    long long k_done = 0;                                           // chunks consumed so far
-    for (long long k = 0; k < n; ++k) {
-        if (tid == 0 && k + kPrefetchA < n) issue(k + kPrefetchA);
-        const int st = (int)(k % kStages);
-        int my_fail = mbar_wait_bounded(&full[st], (phase >> st) & 1u) ? 0 : 1;
-        phase ^= 1u << st;
-        if (!my_fail) {
-            const int cols = chunk_cols(k);
-            const float *sb = ring + (size_t)st * M * CH;
-            float part[M];
-#pragma unroll
-            for (int m = 0; m < M; ++m) part[m] = 0.f;
-            for (int q = tid * 4; q < cols; q += kStagedThreads * 4) {
-                float4 xv[M];
-#pragma unroll
-                for (int m = 0; m < M; ++m) xv[m] = *reinterpret_cast<const float4 *>(sb + m * CH + q);
-                const float4 ebar = shifted_mean<M>(xv);
-#pragma unroll
-                for (int m = 0; m < M; ++m) part[m] = sq_acc(part[m], deviation(xv[m], xv[0], ebar, m));
-            }
-#pragma unroll
-            for (int m = 0; m < M; ++m) acc[m] += (double)part[m];
-        }
-        k_done = k + 1;
-        if (__syncthreads_or(my_fail)) { failed = 1; break; }      // block-uniform decision
-    }
-    if (failed && tid == 0) {
-        // give this block's copies still in flight a bounded chance to land before moving on
-        const long long hi = (k_done - 1 + kPrefetchA < n - 1) ? k_done - 1 + kPrefetchA : n - 1;
-        for (long long k = k_done; k <= hi; ++k) {
-            const int st = (int)(k % kStages);
-            mbar_wait_bounded(&full[st], (phase >> st) & 1u);
-        }
-    }
-    if (blockIdx.x == 0 && tid == 0) {
-        float tail[M];
-#pragma unroll
-        for (int m = 0; m < M; ++m) tail[m] = 0.f;
-        tail_distance<M, false>(a, tail);
-#pragma unroll
-        for (int m = 0; m < M; ++m) acc[m] += (double)tail[m];
-    }
-    {
-        const int lane = tid & 31, warp = tid >> 5;
-#pragma unroll
-        for (int m = 0; m < M; ++m) {
-            double sum = warp_sum(acc[m]);
-            if (lane == 0) s_red[warp * M + m] = sum;
-        }
-        __syncthreads();
-        if (tid < M) {
-            double sum = 0.0;
-            for (int w = 0; w < kStagedWarps; ++w) sum += s_red[w * M + tid];
-            a.partials[(long long)blockIdx.x * M + tid] = failed ? -1.0 : sum;   // negative = "a wait gave up"
-        }
-        if (blockIdx.x == 0 && tid == 0) {
-            a.hdr->status = DPPF_OK;
-            a.hdr->magic = kMagic;
-            a.hdr->grid = (int)gridDim.x;
-            a.hdr->M = M;
-        }
-    }
-    cg::this_grid().sync();
-
-    // ---- every block: did any block give up?  (same answer everywhere)
-    {
-        int bad = 0;
-        for (int i = tid; i < (int)gridDim.x * M; i += kStagedThreads) bad |= (__ldcg(a.partials + i) < 0.0) ? 1 : 0;
-        if (__syncthreads_or(bad)) {
-            if (blockIdx.x == 0 && tid == 0) a.hdr->status = DPPF_ERR_TIMEOUT;
-            return;                                                 // x untouched
-        }
-    }
-    if (!finalise(a, M, (int)gridDim.x, s_c, &s_ok)) return;
-
-    // ---- update pass: local chunks n-1 .. 0; the newest min(n, kStages) are still in the ring
-    const long long resident = (n < kStages) ? n : (long long)kStages;
-    for (long long k = n - 1; k >= 0; --k) {
-        if (tid == 0) {
-            const long long kl = k - kPrefetchB;                    // its stage held chunk kl + kStages: already done
-            if (kl >= 0 && kl < n - resident) issue(kl);
-        }
-        const int st = (int)(k % kStages);
-        int my_fail = 0;
-        if (k < n - resident) {
-            my_fail = mbar_wait_bounded(&full[st], (phase >> st) & 1u) ? 0 : 1;
-            phase ^= 1u << st;
-        }
-        if (!my_fail) {
-            const int cols = chunk_cols(k);
-            const long long c0 = (blockIdx.x + k * gridDim.x) * CH;
-            const float *sb = ring + (size_t)st * M * CH;
-            for (int q = tid * 4; q < cols; q += kStagedThreads * 4) {
-                float4 xv[M];
-#pragma unroll
-                for (int m = 0; m < M; ++m) xv[m] = *reinterpret_cast<const float4 *>(sb + m * CH + q);
-                const float4 ebar = shifted_mean<M>(xv);
-#pragma unroll
-                for (int m = 0; m < M; ++m)
-                    if (row_is_written(s_c[m]))
-                        st_keep(a.x + m * a.ld + c0 + q, apply4(xv[m], deviation(xv[m], xv[0], ebar, m), s_c[m]));
-            }
-        }
-        if (__syncthreads_or(my_fail)) {
-            if (tid == 0) {
-                a.hdr->status = DPPF_ERR_TIMEOUT;                   // x is partly updated
-                const long long kl = k - kPrefetchB;                // the one copy that may still be in flight
-                if (k < n - resident && kl >= 0) mbar_wait_bounded(&full[(int)(kl % kStages)], (phase >> (int)(kl % kStages)) & 1u);
-            }
-            return;
-        }
-    }
-    if (blockIdx.x == 0 && tid == 0) tail_update<M>(a, s_c);
-}
-
-// ---------------------------------------------------------------- general round (staged, M <= 16)
-// Algorithm 1 with an arbitrary consensus variable x_C = sum_m w_m x_m (weights normalised
-// on the host), the push taken from x_A or from x_C (the remark on LSGD), and optionally
-// both terms of the regulariser's gradient (step (a) of the equation in Sec. 5):
-//   y_m  = x_m + alpha (x_C - x_m)                       pull
-//   u_m  = (y_m - P) / ||y_m - P||,  P = x_A or x_C      push direction of the pulled point
-//   x_m+ = y_m + lambda u_m  [ - lambda (1/M) sum_j u_j ]
-// Same two passes and the same traffic as the plain round: on one GPU the mean direction
-// is a per-column register sum, so the second term needs no extra vector or pass.
-// Everything is expressed relative to row 0 (e_m = x_m - x_0), like the shifted mean.
-
-constexpr int kGeneralThreads = 256;   // 384/512/768 threads measured slower (registers)
-constexpr int kGeneralWarps = kGeneralThreads / 32;
-
-struct GeneralArgs {
-    float *x;
-    long long d, ld, nvec;
-    float alpha, lambda;
-    float wn[kMaxTemplateM];     // w_m / sum w
-    int push_from_c, two_term;
-    float *norms_out;            // ||x_m - x_A|| before the round, may be null
-    float *push_norms_out;       // ||y_m - P||, may be null
-    WsHeader *hdr;
-    double *partials;            // [grid][2 M]: squared distances to x_A, then of the pulled points to P
-};
-
-template <int M>
-struct GeneralColumn {
-    // one column: xs[m] in; adds the two squared distances per worker
-    static __device__ __forceinline__ void distances(const float (&xs)[M], const GeneralArgs &a, float (&pr)[M],
-                                                     float (&pn)[M]) {
-        float e[M], ea = 0.f, ec = 0.f;
-        e[0] = 0.f;
-#pragma unroll
-        for (int m = 1; m < M; ++m) {
-            e[m] = __fsub_rn(xs[m], xs[0]);
-            ea = __fadd_rn(ea, e[m]);
-            ec = __fmaf_rn(a.wn[m], e[m], ec);
-        }
-        ea = __fmul_rn(ea, 1.0f / (float)M);
-        const float p = a.push_from_c ? ec : ea;
-#pragma unroll
-        for (int m = 0; m < M; ++m) {
-            const float dev = __fsub_rn(e[m], ea);
-            pr[m] = __fmaf_rn(dev, dev, pr[m]);
-            const float dy = __fmaf_rn(a.alpha, __fsub_rn(ec, e[m]), __fsub_rn(e[m], p));
-            pn[m] = __fmaf_rn(dy, dy, pn[m]);
-        }
-    }
-    // one column: xs[m] in, updated replicas out; g[m] = lambda / ||y_m - P|| (0: no direction)
-    static __device__ __forceinline__ void update(float (&xs)[M], const GeneralArgs &a, const float *g) {
-        float e[M], ea = 0.f, ec = 0.f;
-        e[0] = 0.f;
-#pragma unroll
-        for (int m = 1; m < M; ++m) {
-            e[m] = __fsub_rn(xs[m], xs[0]);
-            ea = __fadd_rn(ea, e[m]);
-            ec = __fmaf_rn(a.wn[m], e[m], ec);
-        }
-        ea = __fmul_rn(ea, 1.0f / (float)M);
-        const float p = a.push_from_c ? ec : ea;
-        float ub = 0.f;                                   // lambda * mean direction
-        if (a.two_term) {
-#pragma unroll
-            for (int m = 0; m < M; ++m) {
-                const float dy = __fmaf_rn(a.alpha, __fsub_rn(ec, e[m]), __fsub_rn(e[m], p));
-                ub = __fmaf_rn(g[m], dy, ub);
-            }
-            ub = __fmul_rn(ub, 1.0f / (float)M);
-        }
-#pragma unroll
-        for (int m = 0; m < M; ++m) {
-            const float pull = __fsub_rn(ec, e[m]);       // x_C - x_m
-            const float dy = __fmaf_rn(a.alpha, pull, __fsub_rn(e[m], p));
-            const float y = __fmaf_rn(a.alpha, pull, xs[m]);
-            xs[m] = __fsub_rn(__fmaf_rn(g[m], dy, y), ub);
-        }
-    }
-};
-
-template <int M>
-__global__ void __launch_bounds__(kGeneralThreads, 1) general_round_kernel(const GeneralArgs a) {
-    constexpr int CH = StagedShape<M>::kChunk;
-    constexpr int kStages = StagedShape<M>::kStages;
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    float *ring = reinterpret_cast<float *>(smem_raw);
-    __shared__ unsigned long long full[kStages];
-    __shared__ double s_red[kGeneralWarps * 2 * M];
-    __shared__ float s_g[M];
-    __shared__ int s_flag;
-    const int tid = threadIdx.x;
-    if (tid == 0) {
-        for (int st = 0; st < kStages; ++st) mbar_init(&full[st], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-
-    const long long d4 = a.nvec * 4;
-    const long long nchunks = (d4 + CH - 1) / CH;
-    const long long n = (nchunks > blockIdx.x) ? (nchunks - 1 - blockIdx.x) / gridDim.x + 1 : 0;
-    unsigned phase = 0;
-    int failed = 0;
-    auto chunk_cols = [&](long long k) -> int {
-        const long long c0 = (blockIdx.x + k * gridDim.x) * CH;
-        return (int)((d4 - c0 < CH) ? (d4 - c0) : CH);
-    };
-    auto issue = [&](long long k) {
-        const int st = (int)(k % kStages);
-        const long long c0 = (blockIdx.x + k * gridDim.x) * CH;
-        const unsigned bytes = (unsigned)chunk_cols(k) * 4u;
-        mbar_expect_tx(&full[st], bytes * M);
-#pragma unroll
-        for (int m = 0; m < M; ++m)
-            bulk_load(ring + ((size_t)st * M + m) * CH, a.x + m * a.ld + c0, bytes, &full[st]);
-    };
-
-    // ---- distance pass: sum (x_m - x_A)^2 and sum (y_m - P)^2 per worker
-    double acc[2 * M];
-#pragma unroll
-    for (int m = 0; m < 2 * M; ++m) acc[m] = 0.0;
-    if (tid == 0)
-        for (long long k = 0; k < kPrefetchA && k < n; ++k) issue(k);
-    long long k_done = 0;
-    for (long long k = 0; k < n; ++k) {
-        if (tid == 0 && k + kPrefetchA < n) issue(k + kPrefetchA);
-        const int st = (int)(k % kStages);
-        int my_fail = mbar_wait_bounded(&full[st], (phase >> st) & 1u) ? 0 : 1;
-        phase ^= 1u << st;
-        if (!my_fail) {
-            const int cols = chunk_cols(k);
-            const float *sb = ring + (size_t)st * M * CH;
-            float pr[M], pn[M];
-#pragma unroll
-            for (int m = 0; m < M; ++m) pr[m] = pn[m] = 0.f;
-            for (int q = tid * 4; q < cols; q += kGeneralThreads * 4) {
-                float4 xv[M];
-#pragma unroll
-                for (int m = 0; m < M; ++m) xv[m] = *reinterpret_cast<const float4 *>(sb + m * CH + q);
-                float xs[M];
-#pragma unroll
-                for (int m = 0; m < M; ++m) xs[m] = xv[m].x;
-                GeneralColumn<M>::distances(xs, a, pr, pn);
-#pragma unroll
-                for (int m = 0; m < M; ++m) xs[m] = xv[m].y;
-                GeneralColumn<M>::distances(xs, a, pr, pn);
-#pragma unroll
-                for (int m = 0; m < M; ++m) xs[m] = xv[m].z;
-                GeneralColumn<M>::distances(xs, a, pr, pn);
-#pragma unroll
-                for (int m = 0; m < M; ++m) xs[m] = xv[m].w;
-                GeneralColumn<M>::distances(xs, a, pr, pn);
-            }
-#pragma unroll
-            for (int m = 0; m < M; ++m) {
-                acc[m] += (double)pr[m];
-                acc[M + m] += (double)pn[m];
-            }
-        }
-        k_done = k + 1;
-        if (__syncthreads_or(my_fail)) { failed = 1; break; }
-    }
-    if (failed && tid == 0) {
-        const long long hi = (k_done - 1 + kPrefetchA < n - 1) ? k_done - 1 + kPrefetchA : n - 1;
-        for (long long k = k_done; k <= hi; ++k) {
-            const int st = (int)(k % kStages);
-            mbar_wait_bounded(&full[st], (phase >> st) & 1u);
-        }
-    }
-    if (blockIdx.x == 0 && tid == 0) {                    // scalar tail columns
-        float pr[M], pn[M];
-#pragma unroll
-        for (int m = 0; m < M; ++m) pr[m] = pn[m] = 0.f;
-        for (long long i = d4; i < a.d; ++i) {
-            float xs[M];
-#pragma unroll
-            for (int m = 0; m < M; ++m) xs[m] = a.x[m * a.ld + i];
-            GeneralColumn<M>::distances(xs, a, pr, pn);
-        }
-#pragma unroll
-        for (int m = 0; m < M; ++m) {
-            acc[m] += (double)pr[m];
-            acc[M + m] += (double)pn[m];
-        }
-    }
-    {
-        const int lane = tid & 31, warp = tid >> 5;
-#pragma unroll
-        for (int m = 0; m < 2 * M; ++m) {
-            double sum = warp_sum(acc[m]);
-            if (lane == 0) s_red[warp * 2 * M + m] = sum;
-        }
-        __syncthreads();
-        if (tid < 2 * M) {
-            double sum = 0.0;
-            for (int w = 0; w < kGeneralWarps; ++w) sum += s_red[w * 2 * M + tid];
-            a.partials[(long long)blockIdx.x * 2 * M + tid] = failed ? -1.0 : sum;
-        }
-        if (blockIdx.x == 0 && tid == 0) {
-            a.hdr->status = DPPF_OK;
-            a.hdr->magic = kMagic;
-            a.hdr->grid = (int)gridDim.x;
-            a.hdr->M = M;
-        }
-    }
-    cg::this_grid().sync();
-
-    {   // did any block give up?
-        int bad = 0;
-        for (int i = tid; i < (int)gridDim.x * 2 * M; i += kGeneralThreads) bad |= (__ldcg(a.partials + i) < 0.0) ? 1 : 0;
-        if (__syncthreads_or(bad)) {
-            if (blockIdx.x == 0 && tid == 0) a.hdr->status = DPPF_ERR_TIMEOUT;
-            return;
-        }
-    }
-    {   // cross-block sums in block order (identical in every block)
-        const int lane = tid & 31, warp = tid >> 5;
-        if (tid == 0) s_flag = 0;
-        __syncthreads();
-        for (int j = warp; j < 2 * M; j += kGeneralWarps) {
-            double sum = 0.0;
-            for (int b = lane; b < (int)gridDim.x; b += 32) sum += __ldcg(a.partials + (long long)b * 2 * M + j);
-            sum = warp_sum(sum);
-            if (lane == 0) {
-                const double nrm = sqrt(sum);
-                if (j < M) {
-                    if (nrm > 0.0) s_flag = 1;            // some replica differs from the average
-                    if (blockIdx.x == 0 && a.norms_out) a.norms_out[j] = (float)nrm;
-                } else {
-                    s_g[j - M] = (nrm > 0.0) ? (float)((double)a.lambda / nrm) : 0.f;
-                    if (blockIdx.x == 0 && a.push_norms_out) a.push_norms_out[j - M] = (float)nrm;
-                }
-            }
-        }
-        __syncthreads();
-        if (!s_flag) return;                              // identical replicas: nothing moves, x untouched
-    }
-
-    // ---- update pass, chunks in reverse, newest chunks reused from the ring
-    const long long resident = (n < kStages) ? n : (long long)kStages;
-    for (long long k = n - 1; k >= 0; --k) {
-        if (tid == 0) {
-            const long long kl = k - kPrefetchB;
-            if (kl >= 0 && kl < n - resident) issue(kl);
-        }
-        const int st = (int)(k % kStages);
-        int my_fail = 0;
-        if (k < n - resident) {
-            my_fail = mbar_wait_bounded(&full[st], (phase >> st) & 1u) ? 0 : 1;
-            phase ^= 1u << st;
-        }
-        if (!my_fail) {
-            const int cols = chunk_cols(k);
-            const long long c0 = (blockIdx.x + k * gridDim.x) * CH;
-            const float *sb = ring + (size_t)st * M * CH;
-            for (int q = tid * 4; q < cols; q += kGeneralThreads * 4) {
-                float4 xv[M];
-#pragma unroll
-                for (int m = 0; m < M; ++m) xv[m] = *reinterpret_cast<const float4 *>(sb + m * CH + q);
-                float xs[M];
-#pragma unroll
-                for (int m = 0; m < M; ++m) xs[m] = xv[m].x;
-                GeneralColumn<M>::update(xs, a, s_g);
-#pragma unroll
-                for (int m = 0; m < M; ++m) { xv[m].x = xs[m]; xs[m] = xv[m].y; }
-                GeneralColumn<M>::update(xs, a, s_g);
-#pragma unroll
-                for (int m = 0; m < M; ++m) { xv[m].y = xs[m]; xs[m] = xv[m].z; }
-                GeneralColumn<M>::update(xs, a, s_g);
-#pragma unroll
-                for (int m = 0; m < M; ++m) { xv[m].z = xs[m]; xs[m] = xv[m].w; }
-                GeneralColumn<M>::update(xs, a, s_g);
-#pragma unroll
-                for (int m = 0; m < M; ++m) {
-                    xv[m].w = xs[m];
-                    st_keep(a.x + m * a.ld + c0 + q, xv[m]);
-                }
-            }
-        }
-        if (__syncthreads_or(my_fail)) {
-            if (tid == 0) {
-                a.hdr->status = DPPF_ERR_TIMEOUT;
-                const long long kl = k - kPrefetchB;
-                if (k < n - resident && kl >= 0) mbar_wait_bounded(&full[(int)(kl % kStages)], (phase >> (int)(kl % kStages)) & 1u);
-            }
-            return;
-        }
-    }
-    if (blockIdx.x == 0 && tid == 0) {
-        for (long long i = d4; i < a.d; ++i) {
-            float xs[M];
-#pragma unroll
-            for (int m = 0; m < M; ++m) xs[m] = a.x[m * a.ld + i];
-            GeneralColumn<M>::update(xs, a, s_g);
-#pragma unroll
-            for (int m = 0; m < M; ++m) a.x[m * a.ld + i] = xs[m];
-        }
-    }
-}
-
-// ---------------------------------------------------------------- generic kernels (16 < M <= 1024)
-// Rows are streamed twice per vector (second time from L1/L2); per-worker sums live in
-// shared memory, one fp32 slot per (warp, worker), so no thread needs M registers.
-
-template <bool kLocalStep>
-__global__ void __launch_bounds__(kThreads) distance_kernel_generic(const RoundArgs a) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    float *s_acc = reinterpret_cast<float *>(smem_raw);               // [kWarps][M]
-    const int M = a.M, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const float inv_m = 1.0f / (float)M;
-    for (int i = threadIdx.x; i < kWarps * M; i += kThreads) s_acc[i] = 0.f;
-    __syncthreads();
-    float *my_acc = s_acc + warp * M;
-    const long long ntiles = (a.nvec + kThreads - 1) / kThreads;
-    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
-        const long long j = t * kThreads + threadIdx.x;
-        const bool live = j < a.nvec;
-        float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), esum = x0;
-        if (live) {
-            for (int m = 0; m < M; ++m) {
-                const long long off = m * a.ld + j * 4;
-                float4 xr = *reinterpret_cast<const float4 *>(a.x + off);
-                if (kLocalStep) {
-                    float4 vr = ld_last_use(a.v + off), gr = ld_last_use(a.g + off);
-                    sgd4(xr, vr, gr, a.lr, a.mu, a.wd);
-                    st_keep(a.v + off, vr);
-                    *reinterpret_cast<float4 *>(a.x + off) = xr;
-                }
-                if (m == 0) x0 = xr; else esum = add4(esum, sub4(xr, x0));
-            }
-        }
-        const float4 ebar = scale4(esum, inv_m);
-        for (int m = 0; m < M; ++m) {
-            float q = 0.f;
-            if (live) {
-                float4 dv;
-                if (m == 0) dv = make_float4(-ebar.x, -ebar.y, -ebar.z, -ebar.w);
-                else dv = sub4(sub4(*reinterpret_cast<const float4 *>(a.x + m * a.ld + j * 4), x0), ebar);
-                q = sq_acc(0.f, dv);
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
-            if (lane == 0) my_acc[m] += q;
-        }
-    }
-    if (blockIdx.x == 0 && threadIdx.x == 0) {      // scalar tail columns
-        for (long long i = a.nvec * 4; i < a.d; ++i) {
-            float x0s = 0.f, esum = 0.f;
-            for (int m = 0; m < M; ++m) {
-                float xi = a.x[m * a.ld + i];
-                if (kLocalStep) {
-                    float vi = a.v[m * a.ld + i];
-                    sgd1(xi, vi, a.g[m * a.ld + i], a.lr, a.mu, a.wd);
-                    a.v[m * a.ld + i] = vi;
-                    a.x[m * a.ld + i] = xi;
-                }
-                if (m == 0) x0s = xi; else esum = __fadd_rn(esum, __fsub_rn(xi, x0s));
-            }
-            const float ebar = __fmul_rn(esum, inv_m);
-            for (int m = 0; m < M; ++m) {
-                float dv = (m == 0) ? -ebar : __fsub_rn(__fsub_rn(a.x[m * a.ld + i], x0s), ebar);
-                my_acc[m] = __fmaf_rn(dv, dv, my_acc[m]);
-            }
-        }
-    }
-    __syncthreads();
-    for (int m = threadIdx.x; m < M; m += kThreads) {
-        double s = 0.0;
-        for (int w = 0; w < kWarps; ++w) s += (double)s_acc[w * M + m];
-        a.partials[(long long)blockIdx.x * M + m] = s;
-    }
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        a.hdr->status = DPPF_OK;
-        a.hdr->magic = kMagic;
-        a.hdr->grid = (int)gridDim.x;
-        a.hdr->M = M;
-    }
-}
-
-__global__ void __launch_bounds__(kThreads) update_kernel_generic(const RoundArgs a, int nblocks_a) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    float *s_c = reinterpret_cast<float *>(smem_raw);                 // [M]
-    __shared__ int s_ok;
-    const int M = a.M;
-    const float inv_m = 1.0f / (float)M;
-    if (!finalise(a, M, nblocks_a, s_c, &s_ok)) return;
-    const long long ntiles = (a.nvec + kThreads - 1) / kThreads;
-    if (ntiles > blockIdx.x) {
-        long long t = blockIdx.x + (ntiles - 1 - blockIdx.x) / gridDim.x * gridDim.x;
-        for (; t >= 0; t -= gridDim.x) {
-            const long long j = t * kThreads + threadIdx.x;
-            if (j >= a.nvec) continue;
-            float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), esum = x0;
-            for (int m = 0; m < M; ++m) {
-                float4 xr = *reinterpret_cast<const float4 *>(a.x + m * a.ld + j * 4);
-                if (m == 0) x0 = xr; else esum = add4(esum, sub4(xr, x0));
-            }
-            const float4 ebar = scale4(esum, inv_m);
-            for (int m = M - 1; m >= 0; --m) {       // row 0 last: the others still need x0 (in a register)
-                float *p = a.x + m * a.ld + j * 4;
-                float4 xr = (m == 0) ? x0 : *reinterpret_cast<const float4 *>(p);
-                float4 dv = (m == 0) ? make_float4(-ebar.x, -ebar.y, -ebar.z, -ebar.w) : sub4(sub4(xr, x0), ebar);
-                if (row_is_written(s_c[m])) st_keep(p, apply4(xr, dv, s_c[m]));
-            }
-        }
-    }
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        for (long long i = a.nvec * 4; i < a.d; ++i) {
-            float x0s = a.x[i], esum = 0.f;
-            for (int m = 1; m < M; ++m) esum = __fadd_rn(esum, __fsub_rn(a.x[m * a.ld + i], x0s));
-            const float ebar = __fmul_rn(esum, inv_m);
-            for (int m = M - 1; m >= 0; --m) {
-                float xi = a.x[m * a.ld + i];
-                float dv = (m == 0) ? -ebar : __fsub_rn(__fsub_rn(xi, x0s), ebar);
-                if (row_is_written(s_c[m])) a.x[m * a.ld + i] = __fmaf_rn(-s_c[m], dv, xi);
-            }
-        }
-    }
-}
-
-// ---------------------------------------------------------------- stand-alone local step
-
-__global__ void __launch_bounds__(kThreads) local_step_kernel(float *x, float *v, const float *g, long long d,
-                                                              long long ld, long long nvec, float lr, float mu,
-                                                              float wd) {
-    const long long row = (long long)blockIdx.y * ld;
-    float *xr = x + row, *vr = v + row;
-    const float *gr = g + row;
-    for (long long j = (long long)blockIdx.x * kThreads + threadIdx.x; j < nvec; j += (long long)gridDim.x * kThreads) {
-        float4 xx = ld_last_use(xr + j * 4), vv = ld_last_use(vr + j * 4), gg = ld_last_use(gr + j * 4);
-        sgd4(xx, vv, gg, lr, mu, wd);
-        st_keep(vr + j * 4, vv);
-        st_keep(xr + j * 4, xx);
-    }
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        for (long long i = nvec * 4; i < d; ++i) {
-            float xi = xr[i], vi = vr[i];
-            sgd1(xi, vi, gr[i], lr, mu, wd);
-            vr[i] = vi;
-            xr[i] = xi;
-        }
-    }
-}
-
-// Zero distances for the one-worker case (x_A == x_1).
-__global__ void zero_norms_kernel(float *norms_out, float *norms_stage, WsHeader *hdr) {
-    if (threadIdx.x == 0) {
-        norms_stage[0] = 0.f;
-        if (norms_out) norms_out[0] = 0.f;
-        hdr->status = DPPF_OK;
-        hdr->magic = 0;
-    }
-}
 
 // ---------------------------------------------------------------- host side
 
