@@ -77,8 +77,9 @@ def workload_of(args):
 
 
 def config_of(w, extra=None):
+    what = ("last local SGD-momentum step fused with the round, steps" if w.tau > 0 else "rounds")
     cfg = {"workload": f"{w.name}: M={w.M} replicas x d={w.d} fp32 ({w.model}), alpha={w.alpha}, lambda={w.lam}, "
-                       f"rounds back to back on one stream",
+                       f"{what} back to back on one stream",
            "M": w.M, "d": w.d, "ld": w.ld, "alpha": w.alpha, "lambda": w.lam,
            "replica_bytes": w.M * w.d * 4,
            "l2_policy": "inputs larger than L2 (no flush between iterations)"}
@@ -189,11 +190,29 @@ def run_reference(args):
     d_s = int(min(w.d, max(4096, rate * per_step * 0.8)))
     ws = w.scaled(d_s)
     x = inputs.replicas(ws, seed)
+    if w.tau > 0:          # local-step workload: one oracle local step, then the round, per step
+        import numpy as np
+        g = inputs.gradients(ws, 0, seed)[:, :d_s]
+        state = {"x": np.ascontiguousarray(x[:, :d_s]), "v": np.zeros((w.M, d_s), dtype=np.float32)}
+
+        def one_step():
+            xo, v64, _ = oracle.local_steps_then_consensus(state["x"], state["v"], [g], w.lr, w.momentum,
+                                                           w.weight_decay, w.alpha, w.lam)
+            state["x"], state["v"] = xo, v64.astype(np.float32)
+        d_s = max(4096, d_s // 8)          # the local step is single-threaded fp64: keep steps short
+        g = np.ascontiguousarray(g[:, :d_s])
+        state = {"x": np.ascontiguousarray(x[:, :d_s]), "v": np.zeros((w.M, d_s), dtype=np.float32)}
+        cores = 1
+    else:
+        state = {"x": x}
+
+        def one_step():
+            state["x"], _, _ = oracle.consensus_blocked(state["x"], w.alpha, w.lam, d=d_s)
     for _ in range(args.warmup):
-        x, _, _ = oracle.consensus_blocked(x, w.alpha, w.lam, d=d_s)
+        one_step()
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        x, _, _ = oracle.consensus_blocked(x, w.alpha, w.lam, d=d_s)
+        one_step()
     dt = (time.perf_counter() - t0) / max(1, args.steps)
     value = 1.0 / (dt * w.d / d_s)
     sample = (f"each step = one oracle round on the first {d_s} of {w.d} columns (all {w.M} rows); "
@@ -268,9 +287,22 @@ def run_ours(args):
     norms = torch.zeros(w.M, device="cuda")
     ws = binding.alloc_workspace(w.M, w.d)
     B = w.M * w.d * 4
+    fused = w.tau > 0          # local-step workload: every step = last local step fused with the round
+    model_units = 7.0 if fused else 3.0      # x M d 4 bytes per step (two-pass fused round: 7, plain round: 3)
+    if fused:
+        v = binding.alloc_rows(w.M, w.d, fill=0.0)
+        g = binding.alloc_rows(w.M, w.d)
+        g.copy_(torch.from_numpy(inputs.gradients(w, 0, seed)).pin_memory(), non_blocking=True)
+        staged = False
+        kernel_name = ("distance_kernel<fused> + update_kernel (one step)" if args.path == "two_kernel" else
+                       "round_kernel<fused> (local step + distance pass, grid barrier, update pass, one launch)")
 
     def step():
-        binding.dppf_consensus(x, w.alpha, w.lam, norms_out=norms, ws=ws, d=w.d, path=path)
+        if fused:
+            binding.dppf_local_step_and_consensus(x, v, g, w.lr, w.momentum, w.weight_decay, w.alpha, w.lam,
+                                                  norms_out=norms, ws=ws, d=w.d, path=path)
+        else:
+            binding.dppf_consensus(x, w.alpha, w.lam, norms_out=norms, ws=ws, d=w.d, path=path)
 
     def fence():
         if world > 1:
@@ -294,12 +326,12 @@ def run_ours(args):
     if binding.dppf_device_status(ws) != binding.OK:
         raise SystemExit("device status word reports an error")
     total_ms = max_over_ranks(total_ms, world, "cuda")
-    launches_per_step = binding.launch_count(w.M, w.d, path)
+    launches_per_step = binding.launch_count(w.M, w.d, path, fused)
 
     # end-to-end: replicas live in pinned host memory; every step copies them in, runs the
     # round and copies the replicas and the M distances back.
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not fused:
         norms_host = torch.zeros(w.M).pin_memory()
         binding.dppf_consensus_host(x_pinned, w.alpha, w.lam, norms_host, x, ws, d=w.d)
         fence()
@@ -316,9 +348,9 @@ def run_ours(args):
 
     if rank == 0:
         peak, peak_src = measured_peaks()
-        achieved = 3.0 * B / (per_launch_ms * 1e-3) / 1e9
+        achieved = model_units * B / (per_launch_ms * 1e-3) / 1e9
         value = whole_job_rate(K, world, total_ms)
-        model_gbs = 3.0 * B * K / (total_ms * 1e-3) / 1e9
+        model_gbs = model_units * B * K / (total_ms * 1e-3) / 1e9
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
                 "warmup": max(3, args.warmup), "ms_per_step": total_ms / K, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
@@ -328,7 +360,7 @@ def run_ours(args):
                 "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                              "frac": achieved / peak, "traffic": measured_traffic(w, staged),
                              "kernel": kernel_name,
-                             "algorithmic_bytes_per_launch": 3 * B, "peak_source": f"of {peak_src}"},
+                             "algorithmic_bytes_per_launch": int(model_units) * B, "peak_source": f"of {peak_src}"},
                 "clocks": clocks.summary(), "gpu_launches": K * launches_per_step,
                 "norms_last_round": [float(v) for v in norms.cpu().tolist()]}
         if e2e is not None:
