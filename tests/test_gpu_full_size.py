@@ -97,3 +97,45 @@ def test_c3_eight_local_steps_then_fused_round(oracle):
     assert_pad_untouched(got_x, w.d), assert_pad_untouched(got_v, w.d)
     # per-element displacement std 0.011053 => r ~ 48.4 (shared start, independent gradients)
     np.testing.assert_allclose(r_ref, 48.4, rtol=0.02)
+
+
+@pytest.mark.parametrize("path", [3, 2])
+def test_rows_longer_than_2_to_31_columns(oracle, path):
+    """64-bit indexing: d = 2^31 + 4099 columns per row (M = 2, 17 GB on the device).  The
+    replicas repeat a random block of P = 2^20 columns, so the CPU oracle can produce the
+    exact answer from one period: sum of squares = (d // P) S_P + S_rest, and the update of a
+    column depends on the other columns only through r_m, which is matched on a slice by
+    rescaling lambda (alpha - lambda'/r_slice = alpha - lambda/r_full)."""
+    import torch
+    _, binding = require_gpu()
+    M, P, d = 2, 1 << 20, (1 << 31) + 4099
+    alpha, lam = 0.1, 0.5
+    rng = np.random.default_rng(41)
+    block = (rng.standard_normal(P)[None, :] * 0.02 + rng.standard_normal((M, P)) * 1e-3).astype(np.float32)
+    reps, rest = divmod(d, P)
+    x = binding.alloc_rows(M, d)
+    blk = torch.from_numpy(block).cuda()
+    x[:, :reps * P].view(M, reps, P).copy_(blk[:, None, :].expand(M, reps, P))
+    x[:, reps * P:d].copy_(blk[:, :rest])
+    x[:, d:].fill_(float("nan"))
+    _, r_p = oracle.consensus(block, alpha, 0.0)
+    _, r_rest = oracle.consensus(np.ascontiguousarray(block[:, :rest]), alpha, 0.0)
+    r_full = np.sqrt(reps * r_p ** 2 + r_rest ** 2)
+    norms = torch.zeros(M, device="cuda")
+    ws = binding.alloc_workspace(M, d)
+    binding.dppf_consensus(x, alpha, lam, norms_out=norms, ws=ws, d=d, path=path)
+    assert binding.dppf_device_status(ws) == binding.OK
+    r = norms.cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(r - r_full) <= 1e-5 * r_full)
+    lam32 = float(np.float32(lam))
+    # the first period, one in the middle, the last whole one (ends at column 2^31) and the
+    # ragged rest beyond 2^31; all of row 1 lies beyond element offset 2^31 as well
+    for start, width, r_slice in ((0, P, r_p), (1000 * P, P, r_p), ((reps - 1) * P, P, r_p),
+                                  (reps * P, rest, r_rest)):
+        ref, _ = oracle.consensus(np.ascontiguousarray(block[:, :width]), alpha, lam32 * r_slice[0] / r_full[0])
+        got = x[:, start:start + width].cpu().numpy()
+        err = np.abs(got.astype(np.float64) - ref)
+        assert np.all(err <= 1e-6 * (1 + np.abs(ref))), (start, float(err.max()))
+    assert torch.isnan(x[:, d:]).all()
+    del x, blk
+    torch.cuda.empty_cache()
