@@ -257,7 +257,7 @@ def run_ours(args):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-    binding.load()
+    binding.load(rebuild_if_stale=True)
     w = workload_of(args)
     seed = (inputs.DEFAULT_SEED if args.seed is None else args.seed) + rank
     path = {"auto": binding.PATH_AUTO, "two_kernel": binding.PATH_TWO_KERNEL,

@@ -8,7 +8,7 @@ def require_gpu():
         import pytest
         pytest.skip("no CUDA device")
     from paper_2507_20424_b200 import binding
-    binding.load()          # raises if the CUDA library is missing: no fallback
+    binding.load(rebuild_if_stale=True)   # compiles with nvcc if needed; raises if it cannot: no fallback
     return torch, binding
 
 
