@@ -28,7 +28,7 @@ def random_replicas(M, d, seed, base=0.02, drift=1e-3):
 
 
 @pytest.mark.parametrize("path", PATHS)
-@pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 7, 8, 16, 17, 40])
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 7, 8, 16, 17, 40, 100])
 @pytest.mark.parametrize("d", [1, 3, 4, 31, 33, 127, 129, 4097, 100_003])
 def test_small_shapes(oracle, M, d, path):
     _, binding = require_gpu()
@@ -50,6 +50,18 @@ def test_workload_recipes_scaled(oracle, name, d, path):
     got, r = gpu_round(binding, x, w.d, w.alpha, w.lam, PATHS[path])
     assert_parity(got, r, ref, r_ref, w.d)
     assert_pad_untouched(got, w.d)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("M,d", [(129, 20_001), (300, 9_999), (1024, 30_003)])
+def test_many_workers(oracle, M, d, path):
+    """Worker counts far beyond the paper's (kernels with per-worker sums in shared memory)."""
+    _, binding = require_gpu()
+    x = random_replicas(M, d, seed=M)
+    ref, r_ref = oracle.consensus(x, 0.1, 0.01, d=d)
+    got, r = gpu_round(binding, x, d, 0.1, 0.01, PATHS[path])
+    assert_parity(got, r, ref, r_ref, d)
+    assert_pad_untouched(got, d)
 
 
 @pytest.mark.parametrize("alpha,lam", [(1.0, 0.0), (0.5, 0.0), (0.0, 0.3), (0.9, 9.0), (0.5, 5.0), (0.05, 0.0)])
@@ -91,7 +103,7 @@ def test_mixed_zero_and_nonzero_distances(oracle):
     assert same_bits(got[0, :50_001], got[1, :50_001]) and same_bits(got[2, :50_001], got[3, :50_001])
 
 
-@pytest.mark.parametrize("M,d", [(4, 3_000_017), (8, 1_000_003), (16, 777_777), (20, 300_001)])
+@pytest.mark.parametrize("M,d", [(4, 3_000_017), (8, 1_000_003), (16, 777_777), (20, 300_001), (64, 150_001)])
 def test_reproducible_and_schedule_independent(M, d):
     """Same input -> same bits run to run for every schedule; the two register schedules
     also agree with each other bit for bit, the staged one to rounding of the distances."""
