@@ -45,6 +45,8 @@ def parse_args():
     p.add_argument("--no-e2e", action="store_true")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--seed", type=int, default=None)
+    p.add_argument("--graph", action="store_true",
+                   help="also time the same steps replayed from a CUDA graph (extra key 'graph_replay')")
     return p.parse_args()
 
 
@@ -328,6 +330,27 @@ def run_ours(args):
     total_ms = max_over_ranks(total_ms, world, "cuda")
     launches_per_step = binding.launch_count(w.M, w.d, path, fused)
 
+    # optional: the same K steps captured once into a CUDA graph and replayed (launch overhead off the host)
+    graph_replay = None
+    if args.graph:
+        chunk = min(K, 100)
+        cg_ = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(cg_):
+            for _ in range(chunk):
+                step()
+        reps = max(1, K // chunk)
+        cg_.replay()
+        fence()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(reps):
+            cg_.replay()
+        g1.record()
+        fence()
+        g_ms = max_over_ranks(g0.elapsed_time(g1), world, "cuda")
+        graph_replay = {"value": whole_job_rate(reps * chunk, world, g_ms), "unit": UNIT,
+                        "steps_per_graph": chunk, "replays": reps, "ms_per_step": g_ms / (reps * chunk)}
+
     # end-to-end: replicas live in pinned host memory; every step copies them in, runs the
     # round and copies the replicas and the M distances back.
     e2e = None
@@ -363,6 +386,8 @@ def run_ours(args):
                              "algorithmic_bytes_per_launch": int(model_units) * B, "peak_source": f"of {peak_src}"},
                 "clocks": clocks.summary(), "gpu_launches": K * launches_per_step,
                 "norms_last_round": [float(v) for v in norms.cpu().tolist()]}
+        if graph_replay is not None:
+            line["graph_replay"] = graph_replay
         if e2e is not None:
             line["e2e"] = e2e
         if cpu is not None:

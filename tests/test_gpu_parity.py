@@ -229,6 +229,32 @@ def test_host_resident_round(oracle):
     assert_pad_untouched(x_host.numpy(), d)
 
 
+def test_rounds_replayed_from_a_cuda_graph_match_eager_rounds():
+    """dppf_consensus launches (cooperative kernels included) can be stream-captured once the
+    first call on the device has been made; a replay gives the eager result bit for bit."""
+    import torch
+    _, binding = require_gpu()
+    d = 1_000_003
+    x_np = random_replicas(4, d, seed=37)
+    ws = binding.alloc_workspace(4, d)
+    norms = torch.zeros(4, device="cuda")
+    eager = to_dev(x_np)
+    for _ in range(5):
+        binding.dppf_consensus(eager, 0.1, 0.005, norms_out=norms, ws=ws, d=d)
+    eager_norms = norms.clone()
+    x = to_dev(x_np)
+    static = x.clone()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(5):
+            binding.dppf_consensus(static, 0.1, 0.005, norms_out=norms, ws=ws, d=d)
+    static.copy_(x)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert same_bits(static.cpu().numpy()[:, :d], eager.cpu().numpy()[:, :d])
+    assert torch.equal(norms, eager_norms)
+
+
 def test_runs_on_a_side_stream(oracle):
     import torch
     _, binding = require_gpu()
