@@ -190,24 +190,22 @@ def run_reference(args):
     _, _, cores = oracle.consensus_blocked(xp, w.alpha, w.lam, d=probe_w.d)
     rate = probe_w.d / max(time.perf_counter() - t0, 1e-6)
     d_s = int(min(w.d, max(4096, rate * per_step * 0.8)))
+    fused = w.tau > 0          # local-step workload: one oracle local step, then the round, per step
+    if fused:
+        d_s = max(4096, d_s // 8)          # the oracle's local step is single-threaded fp64
+        cores = 1
     ws = w.scaled(d_s)
-    x = inputs.replicas(ws, seed)
-    if w.tau > 0:          # local-step workload: one oracle local step, then the round, per step
+    state = {"x": inputs.replicas(ws, seed)}
+    if fused:
         import numpy as np
-        g = inputs.gradients(ws, 0, seed)[:, :d_s]
-        state = {"x": np.ascontiguousarray(x[:, :d_s]), "v": np.zeros((w.M, d_s), dtype=np.float32)}
+        g = np.ascontiguousarray(inputs.gradients(ws, 0, seed)[:, :d_s])
+        state = {"x": np.ascontiguousarray(state["x"][:, :d_s]), "v": np.zeros((w.M, d_s), dtype=np.float32)}
 
         def one_step():
             xo, v64, _ = oracle.local_steps_then_consensus(state["x"], state["v"], [g], w.lr, w.momentum,
                                                            w.weight_decay, w.alpha, w.lam)
             state["x"], state["v"] = xo, v64.astype(np.float32)
-        d_s = max(4096, d_s // 8)          # the local step is single-threaded fp64: keep steps short
-        g = np.ascontiguousarray(g[:, :d_s])
-        state = {"x": np.ascontiguousarray(x[:, :d_s]), "v": np.zeros((w.M, d_s), dtype=np.float32)}
-        cores = 1
     else:
-        state = {"x": x}
-
         def one_step():
             state["x"], _, _ = oracle.consensus_blocked(state["x"], w.alpha, w.lam, d=d_s)
     for _ in range(args.warmup):
@@ -217,7 +215,8 @@ def run_reference(args):
         one_step()
     dt = (time.perf_counter() - t0) / max(1, args.steps)
     value = 1.0 / (dt * w.d / d_s)
-    sample = (f"each step = one oracle round on the first {d_s} of {w.d} columns (all {w.M} rows); "
+    what = "one oracle local step and round" if fused else "one oracle round"
+    sample = (f"each step = {what} on the first {d_s} of {w.d} columns (all {w.M} rows); "
               f"rounds/s scaled by {d_s}/{w.d}")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * w.d / d_s * 1e3,
