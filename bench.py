@@ -98,7 +98,7 @@ class ClockSampler:
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
                0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
 
-    def __init__(self, index, period=0.02):
+    def __init__(self, index, period=0.005):
         self.samples, self.reason_bits, self.max_mhz = [], 0, None
         self._stop = threading.Event()
         self._thread = None
@@ -134,6 +134,10 @@ class ClockSampler:
         self._stop.set()
         if self._thread is not None:
             self._thread.join()
+            try:                      # one more sample while the last launches drain
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+            except Exception:
+                pass
 
     def summary(self):
         if not self.samples:
