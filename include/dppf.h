@@ -13,18 +13,21 @@
  *
  * Conventions for every entry point
  *   - Pointers named x, v, g, norms_out, ws, x_dev are DEVICE pointers owned by the
- *     caller; *_host pointers are HOST pointers.  The library allocates nothing.
+ *     caller; *_host pointers are HOST pointers.  The library allocates nothing
+ *     (dppf_consensus_static keeps its scratch in a fixed array inside the library).
  *   - Layout: row stride ld >= d with ld % 32 == 0, base pointers 128-byte
- *     aligned, so every row starts on a 128-byte boundary.  Columns d..ld-1 are
- *     never read into a result and never written.
+ *     aligned, so every row starts on a 128-byte boundary (a stride that is a
+ *     multiple of 64 floats, i.e. 256 bytes, measures 1-3 % faster).  Columns d..ld-1
+ *     are never read into a result and never written.
  *   - Updates are in place and asynchronous on `cuda_stream` (a cudaStream_t cast
  *     to void*; NULL = the legacy default stream).  Calls that touch the same
  *     buffers or the same workspace must be ordered on one stream.
  *   - x, v and g must not overlap.
  *   - Scalars are fp32 and must be finite; alpha outside (0,1] and negative
  *     lambda are accepted (the invariants alpha = 0 and lambda = 0 need them).
- *   - Return value: a dppf_status.  On any value other than DPPF_OK nothing has
- *     been launched and no buffer has been touched.
+ *   - Return value: a dppf_status.  Arguments are checked before any CUDA call: on
+ *     DPPF_ERR_INVALID_ARG, _ALIGNMENT or _WORKSPACE nothing has been launched and no
+ *     buffer has been touched.
  *   - Zero distance (r_m == 0, e.g. M == 1 or identical replicas): the paper
  *     leaves 0/0 undefined; here no push is applied, the replica is left
  *     bit-for-bit unchanged and r_m = 0 is reported.
