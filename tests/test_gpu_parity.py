@@ -255,6 +255,53 @@ def test_rounds_replayed_from_a_cuda_graph_match_eager_rounds():
     assert torch.equal(norms, eager_norms)
 
 
+def test_random_shapes_and_hyperparameters(oracle):
+    """Eighty seeded random cases over the ranges the paper uses (alpha 0.05..0.9, lambda
+    0.03..90, M 2..16) and a few beyond, every schedule, sizes that straddle tile and chunk
+    boundaries."""
+    _, binding = require_gpu()
+    rng = np.random.default_rng(2507_20424)
+    for case in range(80):
+        M = int(rng.integers(2, 21))
+        d = int(rng.choice([rng.integers(1, 64), rng.integers(64, 5000), rng.integers(5000, 400_000)]))
+        alpha = float(rng.choice([0.05, 0.1, 0.3, 0.5, 0.9, 1.0]))
+        lam = float(rng.choice([0.0, 0.03, 0.1, 0.5, 5.0, 9.0, 90.0]))
+        base = float(rng.choice([0.02, 1.0, 30.0]))
+        drift = base * float(rng.choice([1e-3, 5e-2, 1.0]))
+        x = random_replicas(M, d, seed=1000 + case, base=base, drift=drift)
+        path = int(rng.integers(1, 4))
+        ref, r_ref = oracle.consensus(x, alpha, lam, d=d)
+        got, r = gpu_round(binding, x, d, alpha, lam, path)
+        # fp32 cannot do better than about one ulp of the largest operand (x_m or the step c_m dev_m):
+        # with replicas far apart, or a push much longer than the distances, an updated element can be
+        # much smaller than the terms it is formed from
+        ref64 = ref[:, :d].astype(np.float64)
+        err = np.abs(got[:, :d].astype(np.float64) - ref64)
+        bound = 1e-6 * (1 + np.abs(ref64)) + 1.5e-7 * max(float(np.abs(x[:, :d]).max()), float(np.abs(ref64).max()))
+        info = f"case {case}: M={M} d={d} alpha={alpha} lam={lam} base={base} drift={drift} path={path}"
+        assert np.all(err <= bound), f"{info}: max err {err.max():.3e}"
+        assert np.all(np.abs(r - r_ref) <= 1e-5 * r_ref), info
+        if drift <= 0.05 * base and base <= 1.0 and lam <= 9.0:   # the regime of the workloads: stated tolerance as is
+            assert_parity(got, r, ref, r_ref, d)
+        assert_pad_untouched(got, d)
+
+
+def test_host_resident_round_with_pageable_memory_and_no_norms(oracle):
+    import torch
+    _, binding = require_gpu()
+    d = 123_457
+    x_np = random_replicas(3, d, seed=43)
+    ref, r_ref = oracle.consensus(x_np, 0.3, 0.02, d=d)
+    x_host = torch.from_numpy(x_np.copy())                     # pageable: copies are staged by the driver
+    x_dev = binding.alloc_rows(3, d, fill=float("nan"))
+    ws = binding.alloc_workspace(3, d)
+    binding.dppf_consensus_host(x_host, 0.3, 0.02, None, x_dev, ws, d=d)
+    torch.cuda.synchronize()
+    err = np.abs(x_host.numpy()[:, :d].astype(np.float64) - ref[:, :d])
+    assert np.all(err <= 1e-6 * (1 + np.abs(ref[:, :d])))
+    assert_pad_untouched(x_host.numpy(), d)
+
+
 def test_runs_on_a_side_stream(oracle):
     import torch
     _, binding = require_gpu()
