@@ -81,7 +81,9 @@ int dppf_consensus(float *x, int M, int64_t d, int64_t ld, float alpha, float la
 
 /* Same, with an explicit kernel schedule (DPPF_PATH_*).  Every schedule is reproducible
  * run to run; TWO_KERNEL and COOPERATIVE agree bit for bit, STAGED groups the sums of
- * squares differently and may differ from them in the last bits of r_m. */
+ * squares differently and may differ from them in the last bits of r_m.  If the runtime
+ * refuses a cooperative launch (its blocks cannot all be resident, e.g. SMs shared with
+ * another client) the call falls back to the two-launch schedule. */
 int dppf_consensus_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
                       float *norms_out, void *ws, size_t ws_bytes, int path, void *cuda_stream);
 

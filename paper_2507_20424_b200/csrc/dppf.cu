@@ -128,13 +128,13 @@ int launch_round_m(RoundArgs a, bool fused, int path, int dev, cudaStream_t s) {
             if (grid < 1) grid = 1;
             void *params[] = {&a};
             if (cudaLaunchCooperativeKernel((const void *)round_kernel_staged<M>, dim3((unsigned)grid),
-                                            dim3(kStagedThreads), params, smem, s) != cudaSuccess) {
-                cudaGetLastError();
-                return DPPF_ERR_CUDA;
-            }
-            return DPPF_OK;
+                                            dim3(kStagedThreads), params, smem, s) == cudaSuccess)
+                return DPPF_OK;
+            cudaGetLastError();                         // e.g. not all blocks can be co-resident right now
+            path = DPPF_PATH_TWO_KERNEL;                // (SMs shared with another client): two plain launches
+        } else {
+            path = DPPF_PATH_COOPERATIVE;               // ring does not fit: register kernel instead
         }
-        path = DPPF_PATH_COOPERATIVE;                   // ring does not fit: register kernel instead
     }
     if (path == DPPF_PATH_STAGED) path = DPPF_PATH_COOPERATIVE;
     constexpr int T = Tuning<M>::kThreads;
@@ -162,11 +162,9 @@ int launch_round_m(RoundArgs a, bool fused, int path, int dev, cudaStream_t s) {
     if (path == DPPF_PATH_COOPERATIVE && coop_supported(dev)) {
         void *params[] = {&a};
         const void *fn = fused ? (const void *)round_kernel<M, true> : (const void *)round_kernel<M, false>;
-        if (cudaLaunchCooperativeKernel(fn, dim3((unsigned)grid), dim3(T), params, 0, s) != cudaSuccess) {
-            cudaGetLastError();
-            return DPPF_ERR_CUDA;
-        }
-        return DPPF_OK;
+        if (cudaLaunchCooperativeKernel(fn, dim3((unsigned)grid), dim3(T), params, 0, s) == cudaSuccess)
+            return DPPF_OK;
+        cudaGetLastError();                             // cooperative launch refused: fall back to two launches
     }
     if (fused) {
         distance_kernel<M, true><<<(unsigned)grid, T, 0, s>>>(a);
