@@ -34,6 +34,8 @@ def test_single_round_workloads(oracle, name):
     got, r = _round_on_gpu(binding, x, w)
     assert_parity(got, r, ref, r_ref, w.d)
     assert_pad_untouched(got, w.d)
+    again, r_again = _round_on_gpu(binding, x, w)            # run-to-run reproducible, bit for bit
+    assert same_bits(got[:, :w.d], again[:, :w.d]) and same_bits(r, r_again)
     if name == "C1":       # magnitudes the recipe implies: r_m ~ sigma sqrt(d (M-1)/M)
         np.testing.assert_allclose(r, w.drift_std * np.sqrt(w.d * (w.M - 1) / w.M), rtol=0.01)
 
