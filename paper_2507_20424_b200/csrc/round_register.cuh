@@ -26,7 +26,6 @@ struct Tuning {
     static constexpr int kUnrollFused = 1;
     static constexpr int kUnrollBFused = kUnrollB * (kBlocksPerSM / kBlocksPerSMFused);
     static constexpr int kWarps = kThreads / 32;
-
 };
 
 // Scalar tail: columns 4*nvec .. d-1 (at most three), handled by one thread of block 0.
