@@ -88,6 +88,34 @@ int dppf_consensus_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float
                       float *norms_out, void *ws, size_t ws_bytes, int path, void *cuda_stream);
 
 /*
+ * n_rounds pull-push rounds back to back on x[M, ld], as ONE device pass sequence: the
+ * single-line update of Sec. 5 applied n_rounds times, every round from its own pre-round
+ * average (proof of Theorem 1, first display; the noise-free iteration whose distances the
+ * theorem follows to lambda/alpha).  The result is that of n_rounds calls of
+ * dppf_consensus up to the grouping of the sums of squares (last bits of r_m), but the
+ * update pass of round k also accumulates the squared distances of round k+1 from the values
+ * it has just formed, so the call moves (1 + 2 n_rounds) M d 4 bytes instead of
+ * 3 n_rounds M d 4 and needs one launch per 256 rounds.
+ *   lambdas_host  HOST fp32[n_rounds] with the push strength of every round (e.g. from
+ *                 dppf_lambda_schedule), or NULL: every round uses `lambda`.
+ *   norms_out     NULL, or device fp32[n_rounds, M]: row k receives the distances r_m before
+ *                 round k (the per-round consensus distances the ablations plot).
+ * Workspace and layout rules as for dppf_consensus.  M <= 16 runs the fused schedule; M = 1 and
+ * M > 16, and any M when the runtime refuses a cooperative launch, run one round per launch
+ * instead (same results, 3 M d 4 bytes per round).  The _ex form selects the kernel family:
+ * DPPF_PATH_STAGED (default for M <= 8), DPPF_PATH_COOPERATIVE (register kernel, default
+ * for 9 <= M <= 16), DPPF_PATH_TWO_KERNEL (one round per call of dppf_consensus_ex).
+ * If a bounded wait gives up (dppf_device_status: DPPF_ERR_TIMEOUT) x is untouched when that
+ * happened before the first update and holds a mixture of rounds otherwise.
+ */
+int dppf_consensus_rounds(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
+                          const float *lambdas_host, int n_rounds, float *norms_out, void *ws,
+                          size_t ws_bytes, void *cuda_stream);
+int dppf_consensus_rounds_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
+                             const float *lambdas_host, int n_rounds, float *norms_out, void *ws,
+                             size_t ws_bytes, int path, void *cuda_stream);
+
+/*
  * General consensus round (Algorithm 1 with an arbitrary consensus variable; Sec. 5,
  * step (a) of the regulariser-gradient equation; the remark on LSGD in the appendix):
  *   x_C  = sum_m w_m x_m / sum_m w_m      weights_host: HOST fp32[M], NULL = all equal (x_C = x_A);
@@ -239,6 +267,19 @@ int dppf_round_metrics(const float *norms_host, int M, float alpha, float lambda
  * updated otherwise).  DPPF_ERR_CUDA if the stream failed.
  */
 int dppf_device_status(const void *ws, void *cuda_stream);
+
+/*
+ * Testing hook (the paper has no counterpart).  The kernels that stage rows through shared
+ * memory wait for their asynchronous copies with a bounded number of polls (default 2^22,
+ * about a second) and report DPPF_ERR_TIMEOUT through the status word if a wait runs out.
+ * This sets the poll budget of later calls in this process: first_pass_polls for waits of the
+ * distance pass, later_pass_polls for waits of update passes; a negative value restores the
+ * default.  A budget of 0 makes every such wait give up at once while the copies themselves
+ * still complete (the block waits for them with the full budget before it leaves), which is
+ * how the tests drive the give-up path on a healthy GPU.  Applies to dppf_consensus_rounds,
+ * dppf_consensus (staged schedule) and dppf_consensus_general.  Always returns DPPF_OK.
+ */
+int dppf_debug_set_poll_limits(int first_pass_polls, int later_pass_polls);
 
 /* Static, human-readable name of a dppf_status. */
 const char *dppf_status_string(int status);

@@ -21,6 +21,7 @@ EXPORTS = ("dppf_workspace_bytes", "dppf_consensus", "dppf_consensus_ex", "dppf_
            "dppf_local_step_and_consensus", "dppf_local_step_and_consensus_ex",
            "dppf_consensus_host", "dppf_device_status", "dppf_status_string", "dppf_launch_count",
            "dppf_consensus_static", "dppf_consensus_general",
+           "dppf_consensus_rounds", "dppf_consensus_rounds_ex", "dppf_debug_set_poll_limits",
            "dppf_adamw_step", "dppf_adamw_step_and_consensus",
            "dppf_lambda_schedule", "dppf_lr_cosine", "dppf_qsr_period", "dppf_round_metrics")
 
@@ -75,6 +76,13 @@ def load(rebuild_if_stale: bool = False) -> ctypes.CDLL:
     lib.dppf_consensus_general.argtypes = [vp, i32, i64, i64, f32, f32, ctypes.POINTER(f32), i32, i32, vp, vp,
                                            vp, sz, vp]
     lib.dppf_consensus_general.restype = i32
+    lib.dppf_consensus_rounds.argtypes = [vp, i32, i64, i64, f32, f32, ctypes.POINTER(f32), i32, vp, vp, sz, vp]
+    lib.dppf_consensus_rounds.restype = i32
+    lib.dppf_consensus_rounds_ex.argtypes = [vp, i32, i64, i64, f32, f32, ctypes.POINTER(f32), i32, vp, vp, sz,
+                                             i32, vp]
+    lib.dppf_consensus_rounds_ex.restype = i32
+    lib.dppf_debug_set_poll_limits.argtypes = [i32, i32]
+    lib.dppf_debug_set_poll_limits.restype = i32
     lib.dppf_consensus_static.argtypes = [vp, i32, i64, i64, f32, f32, vp, vp]
     lib.dppf_consensus_static.restype = i32
     lib.dppf_status_string.argtypes = [i32]
@@ -140,6 +148,29 @@ def dppf_consensus(x, alpha, lam, norms_out=None, ws=None, d=None, path=PATH_AUT
                                   ws.data_ptr(), ws.numel(), int(path), _stream())
     _check(rc, "dppf_consensus")
     return ws
+
+
+def dppf_consensus_rounds(x, alpha, lam, n_rounds, lambdas=None, norms_out=None, ws=None, d=None, path=PATH_AUTO):
+    """``n_rounds`` rounds in place on ``x[M, ld]`` in one pass sequence; ``lambdas`` (host
+    sequence of n_rounds floats) overrides ``lam`` per round; ``norms_out`` is [n_rounds, M]."""
+    M, d, ld = _dims(x, d)
+    ws = alloc_workspace(M, d, x.device) if ws is None else ws
+    lp = None
+    if lambdas is not None:
+        if len(lambdas) != n_rounds:
+            raise ValueError("lambdas must have one entry per round")
+        lp = (ctypes.c_float * n_rounds)(*[float(v) for v in lambdas])
+    if norms_out is not None and norms_out.numel() < n_rounds * M:
+        raise ValueError("norms_out must hold n_rounds x M floats")
+    rc = load().dppf_consensus_rounds_ex(x.data_ptr(), M, d, ld, alpha, lam, lp, int(n_rounds), _ptr(norms_out),
+                                         ws.data_ptr(), ws.numel(), int(path), _stream())
+    _check(rc, "dppf_consensus_rounds")
+    return ws
+
+
+def debug_set_poll_limits(first_pass_polls=-1, later_pass_polls=-1) -> None:
+    """Testing hook: poll budget of the bounded waits of later calls (negative = default)."""
+    load().dppf_debug_set_poll_limits(int(first_pass_polls), int(later_pass_polls))
 
 
 PUSH_FROM_AVERAGE, PUSH_FROM_CONSENSUS = 0, 1

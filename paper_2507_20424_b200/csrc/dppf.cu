@@ -4,6 +4,7 @@
 //   round_register.cuh  register-resident round kernels (two-launch and cooperative schedules)
 //   adamw.cuh           AdamW local step, stand-alone and fused into the distance pass
 //   round_staged.cuh    staged persistent round kernel (bulk async copies into a shared-memory ring)
+//   round_multi.cuh     several rounds in one launch (update pass of round k + distances of round k+1)
 //   round_general.cuh   general round (weighted consensus variable, push reference, two-term push)
 //   round_generic.cuh   any worker count up to 1024, stand-alone SGD-momentum local step
 //
@@ -33,6 +34,7 @@
 #include "round_register.cuh"
 #include "adamw.cuh"
 #include "round_staged.cuh"
+#include "round_multi.cuh"
 #include "round_general.cuh"
 #include "round_generic.cuh"
 
@@ -299,6 +301,84 @@ int static_ws_address(int dev, void **out) {
 }
 
 
+// ---------------------------------------------------------------- several rounds per launch: host side
+// Poll limits of the bounded waits (first pass / later passes).  Only the testing hook
+// dppf_debug_set_poll_limits changes them.
+std::atomic<int> g_spin_first{kSpinLimit}, g_spin_later{kSpinLimit};
+std::atomic<int> g_rounds_ready[64][kMaxTemplateM + 1][2];   // [][][0] staged, [1] register: blocks per SM
+
+// One launch of up to kMaxRoundsPerLaunch rounds.  DPPF_ERR_CUDA + *refused = true when the
+// runtime will not launch cooperatively (caller falls back to single rounds).
+template <int M>
+int launch_rounds_m(RoundsArgs &a, int path, int dev, cudaStream_t s, bool *refused) {
+    *refused = false;
+    const int sms = sm_count(dev);
+    if (sms <= 0) return DPPF_ERR_CUDA;
+    if (!coop_supported(dev)) { *refused = true; return DPPF_ERR_CUDA; }
+    void *params[] = {&a};
+    if (path == DPPF_PATH_STAGED) {
+        constexpr size_t smem = StagedShape<M>::kSmemBytes;
+        if (g_rounds_ready[dev][M][0].load(std::memory_order_relaxed) == 0) {
+            int n = 0;
+            if (cudaFuncSetAttribute(rounds_kernel_staged<M>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)smem) != cudaSuccess ||
+                cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, rounds_kernel_staged<M>, kStagedThreads, smem) !=
+                    cudaSuccess || n < 1) {
+                cudaGetLastError();
+                *refused = true;
+                return DPPF_ERR_CUDA;
+            }
+            g_rounds_ready[dev][M][0].store(n, std::memory_order_relaxed);
+        }
+        const long long nchunks = (a.nvec * 4 + StagedShape<M>::kChunk - 1) / StagedShape<M>::kChunk;
+        long long grid = sms;                           // one block per SM
+        if (grid > nchunks) grid = nchunks;
+        if (grid > kMaxBlocksSmallM / 2) grid = kMaxBlocksSmallM / 2;
+        if (grid < 1) grid = 1;
+        if (cudaLaunchCooperativeKernel((const void *)rounds_kernel_staged<M>, dim3((unsigned)grid),
+                                        dim3(kStagedThreads), params, smem, s) == cudaSuccess)
+            return DPPF_OK;
+        cudaGetLastError();
+        *refused = true;
+        return DPPF_ERR_CUDA;
+    }
+    constexpr int T = Tuning<M>::kThreads;
+    int per_sm = g_rounds_ready[dev][M][1].load(std::memory_order_relaxed);
+    if (per_sm == 0) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rounds_kernel<M>, T, 0) != cudaSuccess ||
+            per_sm < 1) {
+            cudaGetLastError();
+            *refused = true;
+            return DPPF_ERR_CUDA;
+        }
+        g_rounds_ready[dev][M][1].store(per_sm, std::memory_order_relaxed);
+    }
+    if (per_sm > Tuning<M>::kBlocksPerSM) per_sm = Tuning<M>::kBlocksPerSM;
+    const int u = Tuning<M>::kUnrollA > Tuning<M>::kUnrollB ? Tuning<M>::kUnrollA : Tuning<M>::kUnrollB;
+    long long ntiles = (a.nvec + (long long)T * u - 1) / ((long long)T * u);
+    long long grid = (long long)sms * per_sm;
+    if (grid > ntiles) grid = ntiles;
+    if (grid > kMaxBlocksSmallM / 2) grid = kMaxBlocksSmallM / 2;
+    if (grid < 1) grid = 1;
+    if (cudaLaunchCooperativeKernel((const void *)rounds_kernel<M>, dim3((unsigned)grid), dim3(T), params, 0, s) ==
+        cudaSuccess)
+        return DPPF_OK;
+    cudaGetLastError();
+    *refused = true;
+    return DPPF_ERR_CUDA;
+}
+
+int launch_rounds(RoundsArgs &a, int M, int path, int dev, cudaStream_t s, bool *refused) {
+    switch (M) {
+#define DPPF_CASE(MM) case MM: return launch_rounds_m<MM>(a, path, dev, s, refused);
+        DPPF_CASE(2) DPPF_CASE(3) DPPF_CASE(4) DPPF_CASE(5) DPPF_CASE(6) DPPF_CASE(7) DPPF_CASE(8)
+        DPPF_CASE(9) DPPF_CASE(10) DPPF_CASE(11) DPPF_CASE(12) DPPF_CASE(13) DPPF_CASE(14) DPPF_CASE(15)
+        DPPF_CASE(16)
+#undef DPPF_CASE
+        default: *refused = true; return DPPF_ERR_CUDA;
+    }
+}
+
 // ---------------------------------------------------------------- general round: host side
 std::atomic<int> g_general_ready[64][kMaxTemplateM + 1];
 
@@ -497,6 +577,76 @@ int dppf_launch_count(int M, int64_t d, int path, int fused) {
     if (M < 1 || M > DPPF_MAX_WORKERS || d < 1) return 0;
     if (M == 1) return fused ? 2 : 1;                       // [local step], zero norms
     return resolve_path(path, M, fused != 0) == DPPF_PATH_TWO_KERNEL ? 2 : 1;
+}
+
+int dppf_consensus_rounds_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
+                             const float *lambdas_host, int n_rounds, float *norms_out, void *ws, size_t ws_bytes,
+                             int path, void *cuda_stream) {
+    int rc = check_layout(x, M, d, ld);
+    if (rc != DPPF_OK) return rc;
+    if (n_rounds < 1) return DPPF_ERR_INVALID_ARG;
+    if (path != DPPF_PATH_AUTO && path != DPPF_PATH_TWO_KERNEL && path != DPPF_PATH_COOPERATIVE &&
+        path != DPPF_PATH_STAGED)
+        return DPPF_ERR_INVALID_ARG;
+    if (!finite_all({alpha})) return DPPF_ERR_INVALID_ARG;
+    if (lambdas_host) {
+        for (int k = 0; k < n_rounds; ++k)
+            if (!std::isfinite(lambdas_host[k])) return DPPF_ERR_INVALID_ARG;
+    } else if (!finite_all({lambda})) {
+        return DPPF_ERR_INVALID_ARG;
+    }
+    if (!ws) return DPPF_ERR_INVALID_ARG;
+    if (!aligned128(ws)) return DPPF_ERR_ALIGNMENT;
+    if (ws_bytes < workspace_bytes(M)) return DPPF_ERR_WORKSPACE;
+    const size_t bytes = (size_t)M * (size_t)ld * sizeof(float);
+    if (overlap(x, bytes, ws, workspace_bytes(M))) return DPPF_ERR_INVALID_ARG;
+    if (norms_out && overlap(x, bytes, norms_out, (size_t)n_rounds * M * sizeof(float))) return DPPF_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DPPF_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+
+    if (path == DPPF_PATH_AUTO) path = (M <= 8) ? DPPF_PATH_STAGED : DPPF_PATH_COOPERATIVE;
+    bool single_rounds = (M == 1 || M > kMaxTemplateM || path == DPPF_PATH_TWO_KERNEL);
+    int done = 0;
+    while (!single_rounds && done < n_rounds) {
+        RoundsArgs a;
+        a.x = x; a.d = d; a.ld = ld; a.nvec = d / 4;
+        a.alpha = alpha;
+        a.n_rounds = (n_rounds - done < kMaxRoundsPerLaunch) ? n_rounds - done : kMaxRoundsPerLaunch;
+        a.spin_first = g_spin_first.load(std::memory_order_relaxed);
+        a.spin_later = g_spin_later.load(std::memory_order_relaxed);
+        a.norms_all = norms_out ? norms_out + (size_t)done * M : nullptr;
+        a.norms_stage = reinterpret_cast<float *>(static_cast<unsigned char *>(ws) + norms_stage_offset(M));
+        a.hdr = reinterpret_cast<WsHeader *>(ws);
+        a.partials = reinterpret_cast<double *>(static_cast<unsigned char *>(ws) + kHeaderBytes);
+        a.partials_half = (long long)(kMaxBlocksSmallM / 2) * M;
+        for (int k = 0; k < a.n_rounds; ++k) a.lambdas[k] = lambdas_host ? lambdas_host[done + k] : lambda;
+        bool refused = false;
+        rc = launch_rounds(a, M, path, dev, s, &refused);
+        if (rc == DPPF_OK) { done += a.n_rounds; continue; }
+        if (!refused) return rc;
+        single_rounds = true;       // cooperative launch not possible right now: one round per call below
+    }
+    for (; done < n_rounds; ++done) {
+        rc = run_round(x, nullptr, nullptr, M, d, ld, 0.f, 0.f, 0.f, alpha, lambdas_host ? lambdas_host[done] : lambda,
+                       norms_out ? norms_out + (size_t)done * M : nullptr, ws, ws_bytes,
+                       path == DPPF_PATH_TWO_KERNEL ? DPPF_PATH_TWO_KERNEL : DPPF_PATH_AUTO, false, s);
+        if (rc != DPPF_OK) return rc;
+    }
+    return DPPF_OK;
+}
+
+int dppf_consensus_rounds(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
+                          const float *lambdas_host, int n_rounds, float *norms_out, void *ws, size_t ws_bytes,
+                          void *cuda_stream) {
+    return dppf_consensus_rounds_ex(x, M, d, ld, alpha, lambda, lambdas_host, n_rounds, norms_out, ws, ws_bytes,
+                                    DPPF_PATH_AUTO, cuda_stream);
+}
+
+int dppf_debug_set_poll_limits(int first_pass_polls, int later_pass_polls) {
+    g_spin_first.store(first_pass_polls < 0 ? kSpinLimit : first_pass_polls, std::memory_order_relaxed);
+    g_spin_later.store(later_pass_polls < 0 ? kSpinLimit : later_pass_polls, std::memory_order_relaxed);
+    return DPPF_OK;
 }
 
 int dppf_consensus_static(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda, float *norms_out,

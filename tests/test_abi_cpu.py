@@ -94,6 +94,15 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert gen(X, 4, 64, 64, 0.1, 0.01, w_zero, 0, 0, None, None, WS, big, None) == b.ERR_INVALID_ARG
     assert gen(X, 4, 64, 64, 0.1, 0.01, w_ok, 0, 1, None, None, WS, 16, None) == b.ERR_WORKSPACE
     assert gen(X, 4, 60, 60, 0.1, 0.01, w_ok, 0, 1, None, None, WS, big, None) == b.ERR_ALIGNMENT
+    rounds = lib.dppf_consensus_rounds
+    lam_bad = (ctypes.c_float * 2)(0.1, float("inf"))
+    assert rounds(None, 4, 64, 64, 0.1, 0.01, None, 3, None, WS, big, None) == b.ERR_INVALID_ARG
+    assert rounds(X, 4, 64, 64, 0.1, 0.01, None, 0, None, WS, big, None) == b.ERR_INVALID_ARG
+    assert rounds(X, 4, 64, 64, 0.1, 0.01, lam_bad, 2, None, WS, big, None) == b.ERR_INVALID_ARG
+    assert rounds(X, 4, 64, 64, float("nan"), 0.01, None, 2, None, WS, big, None) == b.ERR_INVALID_ARG
+    assert rounds(X, 4, 64, 64, 0.1, 0.01, None, 2, None, WS, 16, None) == b.ERR_WORKSPACE
+    assert rounds(X, 4, 64, 64, 0.1, 0.01, None, 2, X + 64, WS, big, None) == b.ERR_INVALID_ARG   # norms inside x
+    assert lib.dppf_consensus_rounds_ex(X, 4, 64, 64, 0.1, 0.01, None, 2, None, WS, big, 9, None) == b.ERR_INVALID_ARG
 
 
 def test_binding_refuses_cpu_tensors(lib):
