@@ -61,7 +61,7 @@ typedef enum {
 #define DPPF_PATH_TWO_KERNEL 1  /* distance pass, then update pass, as two launches */
 #define DPPF_PATH_COOPERATIVE 2 /* one persistent cooperative launch with a grid-wide barrier */
 #define DPPF_PATH_STAGED 3      /* cooperative launch, rows staged through shared memory by bulk
-                                   async copies; what AUTO picks for dppf_consensus when M <= 8 */
+                                   async copies; what AUTO picks for dppf_consensus when M <= 16 */
 
 /*
  * Scratch size in bytes for a round on M replicas of length d (the per-block
@@ -103,8 +103,8 @@ int dppf_consensus_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float
  * Workspace and layout rules as for dppf_consensus.  M <= 16 runs the fused schedule; M = 1 and
  * M > 16, and any M when the runtime refuses a cooperative launch, run one round per launch
  * instead (same results, 3 M d 4 bytes per round).  The _ex form selects the kernel family:
- * DPPF_PATH_STAGED (default for M <= 8), DPPF_PATH_COOPERATIVE (register kernel, default
- * for 9 <= M <= 16), DPPF_PATH_TWO_KERNEL (one round per call of dppf_consensus_ex).
+ * DPPF_PATH_STAGED (default), DPPF_PATH_COOPERATIVE (register kernel),
+ * DPPF_PATH_TWO_KERNEL (one round per call of dppf_consensus_ex).
  * If a bounded wait gives up (dppf_device_status: DPPF_ERR_TIMEOUT) x is untouched when that
  * happened before the first update and holds a mixture of rounds otherwise.
  */
@@ -114,6 +114,28 @@ int dppf_consensus_rounds(float *x, int M, int64_t d, int64_t ld, float alpha, f
 int dppf_consensus_rounds_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
                              const float *lambdas_host, int n_rounds, float *norms_out, void *ws,
                              size_t ws_bytes, int path, void *cuda_stream);
+
+/*
+ * One round split at its reduction, for replicas whose COLUMNS are sharded over several GPUs
+ * (each GPU holds x[M, d_g]: all M workers, a slice of the parameters).  In Algorithm 1 the
+ * workers meet once per round to "obtain x_C"; with column shards the average of a column is
+ * local to the GPU that holds it, and what has to be exchanged instead is the M sums of squares
+ * behind the norms ||x_m - x_A|| of the single-line update (Sec. 5):
+ *   dppf_distance_partials   sums_out[m] = sum over this shard's columns of (x_m - x_A)^2
+ *                            (device fp64[M]; deterministic: fixed block order);
+ *   -- the caller adds the M doubles over all shards (e.g. an all-reduce) --
+ *   dppf_update_from_sums    r_m = sqrt(sums[m]), c_m = alpha - lambda / r_m, then the update
+ *                            x_m <- x_m + (x_A - x_m) c_m on this shard (sums: device fp64[M],
+ *                            the TOTALS over all shards; norms_out: NULL or device fp32[M], r_m).
+ * With one shard the pair equals dppf_consensus (two-launch schedule) bit for bit.  A worker
+ * with sums[m] == 0 is left untouched.  dppf_distance_partials reads x only; its workspace is
+ * that of dppf_consensus.  dppf_update_from_sums needs no workspace.  Any M <= DPPF_MAX_WORKERS.
+ * A shard may be a column range of a wider buffer (pointer x + first column, same ld).
+ */
+int dppf_distance_partials(const float *x, int M, int64_t d, int64_t ld, double *sums_out, void *ws,
+                           size_t ws_bytes, void *cuda_stream);
+int dppf_update_from_sums(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
+                          const double *sums, float *norms_out, void *cuda_stream);
 
 /*
  * General consensus round (Algorithm 1 with an arbitrary consensus variable; Sec. 5,
@@ -129,7 +151,9 @@ int dppf_consensus_rounds_ex(float *x, int M, int64_t d, int64_t ld, float alpha
  *                                         the gradient of the relaxed Inverse-Mean-Valley
  *                                         regulariser, lambda = lambda_r / M
  * x_A, x_C and P are the pre-round values for every worker.  A worker whose pulled point
- * equals P has no direction and is not pushed.  With weights_host == NULL, push from the
+ * equals P has no direction and is not pushed (with equal weights x_C is x_A bit for bit, so
+ * alpha = 1 with the push taken from the average puts every replica on x_A, to fp32 rounding,
+ * and reports zero push distances).  With weights_host == NULL, push from the
  * average, two_term == 0 and alpha < 1 this is dppf_consensus.  Identical replicas are left
  * untouched.  M <= 16.  norms_out (device fp32[M] or NULL) receives ||x_m - x_A|| before the
  * round, push_norms_out (device fp32[M] or NULL) receives ||y_m - P||.  Workspace and layout
@@ -141,6 +165,14 @@ int dppf_consensus_general(float *x, int M, int64_t d, int64_t ld, float alpha, 
                            const float *weights_host, int push_from, int two_term,
                            float *norms_out, float *push_norms_out, void *ws, size_t ws_bytes,
                            void *cuda_stream);
+/* Same with an explicit schedule: DPPF_PATH_AUTO or DPPF_PATH_STAGED (one cooperative launch,
+ * rows staged through shared memory; falls back to two launches if the runtime refuses it) or
+ * DPPF_PATH_TWO_KERNEL (distance launch, then update launch, register kernels).  The two
+ * schedules group the sums of squares differently (last bits of the distances). */
+int dppf_consensus_general_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
+                              const float *weights_host, int push_from, int two_term,
+                              float *norms_out, float *push_norms_out, void *ws, size_t ws_bytes,
+                              int path, void *cuda_stream);
 
 /*
  * One local optimiser step between rounds, in place, for all M workers
@@ -189,6 +221,14 @@ int dppf_adamw_step_and_consensus(float *x, float *exp_avg, float *exp_avg_sq, c
                                   int64_t d, int64_t ld, float lr, float beta1, float beta2, float eps,
                                   float weight_decay, int step, float alpha, float lambda,
                                   float *norms_out, void *ws, size_t ws_bytes, void *cuda_stream);
+/* Same with an explicit schedule: DPPF_PATH_AUTO / DPPF_PATH_COOPERATIVE (one persistent launch:
+ * step + distance pass, grid barrier, update pass; falls back to two launches if the runtime
+ * refuses it) or DPPF_PATH_TWO_KERNEL.  Both schedules use the same grid and agree bit for bit. */
+int dppf_adamw_step_and_consensus_ex(float *x, float *exp_avg, float *exp_avg_sq, const float *g, int M,
+                                     int64_t d, int64_t ld, float lr, float beta1, float beta2, float eps,
+                                     float weight_decay, int step, float alpha, float lambda,
+                                     float *norms_out, void *ws, size_t ws_bytes, int path,
+                                     void *cuda_stream);
 
 /*
  * Round on replicas that live in HOST memory (the arrangement the paper's
@@ -232,6 +272,9 @@ int dppf_consensus_host(float *x_host, int M, int64_t d, int64_t ld, float alpha
 #define DPPF_STATIC_MAX_WORKERS 16
 int dppf_consensus_static(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
                           float *norms_out, void *cuda_stream);
+/* dppf_device_status for the built-in scratch of the current device: a caller of
+ * dppf_consensus_static has no workspace pointer to pass.  Synchronises `cuda_stream`. */
+int dppf_static_device_status(void *cuda_stream);
 
 /*
  * Host-side scalars of a DPPF run (no device work, no CUDA call).
@@ -277,7 +320,8 @@ int dppf_device_status(const void *ws, void *cuda_stream);
  * default.  A budget of 0 makes every such wait give up at once while the copies themselves
  * still complete (the block waits for them with the full budget before it leaves), which is
  * how the tests drive the give-up path on a healthy GPU.  Applies to dppf_consensus_rounds,
- * dppf_consensus (staged schedule) and dppf_consensus_general.  Always returns DPPF_OK.
+ * dppf_consensus and dppf_consensus_static (staged schedule) and dppf_consensus_general.
+ * Always returns DPPF_OK.
  */
 int dppf_debug_set_poll_limits(int first_pass_polls, int later_pass_polls);
 
@@ -285,7 +329,7 @@ int dppf_debug_set_poll_limits(int first_pass_polls, int later_pass_polls);
 const char *dppf_status_string(int status);
 
 /* Number of kernel launches the given call shape issues (for launch accounting):
- * fused != 0 selects dppf_local_step_and_consensus. */
+ * fused == 0 dppf_consensus_ex, 1 dppf_local_step_and_consensus_ex, 2 dppf_adamw_step_and_consensus_ex. */
 int dppf_launch_count(int M, int64_t d, int path, int fused);
 
 #ifdef __cplusplus

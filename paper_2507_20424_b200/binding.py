@@ -20,7 +20,8 @@ OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range
 EXPORTS = ("dppf_workspace_bytes", "dppf_consensus", "dppf_consensus_ex", "dppf_local_step",
            "dppf_local_step_and_consensus", "dppf_local_step_and_consensus_ex",
            "dppf_consensus_host", "dppf_device_status", "dppf_status_string", "dppf_launch_count",
-           "dppf_consensus_static", "dppf_consensus_general",
+           "dppf_consensus_static", "dppf_static_device_status", "dppf_consensus_general", "dppf_consensus_general_ex",
+           "dppf_distance_partials", "dppf_update_from_sums", "dppf_adamw_step_and_consensus_ex",
            "dppf_consensus_rounds", "dppf_consensus_rounds_ex", "dppf_debug_set_poll_limits",
            "dppf_adamw_step", "dppf_adamw_step_and_consensus",
            "dppf_lambda_schedule", "dppf_lr_cosine", "dppf_qsr_period", "dppf_round_metrics")
@@ -81,6 +82,18 @@ def load(rebuild_if_stale: bool = False) -> ctypes.CDLL:
     lib.dppf_consensus_rounds_ex.argtypes = [vp, i32, i64, i64, f32, f32, ctypes.POINTER(f32), i32, vp, vp, sz,
                                              i32, vp]
     lib.dppf_consensus_rounds_ex.restype = i32
+    lib.dppf_distance_partials.argtypes = [vp, i32, i64, i64, vp, vp, sz, vp]
+    lib.dppf_distance_partials.restype = i32
+    lib.dppf_update_from_sums.argtypes = [vp, i32, i64, i64, f32, f32, vp, vp, vp]
+    lib.dppf_update_from_sums.restype = i32
+    lib.dppf_static_device_status.argtypes = [vp]
+    lib.dppf_static_device_status.restype = i32
+    lib.dppf_consensus_general_ex.argtypes = [vp, i32, i64, i64, f32, f32, ctypes.POINTER(f32), i32, i32, vp, vp,
+                                              vp, sz, i32, vp]
+    lib.dppf_consensus_general_ex.restype = i32
+    lib.dppf_adamw_step_and_consensus_ex.argtypes = [vp, vp, vp, vp, i32, i64, i64, f32, f32, f32, f32, f32, i32,
+                                                     f32, f32, vp, vp, sz, i32, vp]
+    lib.dppf_adamw_step_and_consensus_ex.restype = i32
     lib.dppf_debug_set_poll_limits.argtypes = [i32, i32]
     lib.dppf_debug_set_poll_limits.restype = i32
     lib.dppf_consensus_static.argtypes = [vp, i32, i64, i64, f32, f32, vp, vp]
@@ -168,6 +181,27 @@ def dppf_consensus_rounds(x, alpha, lam, n_rounds, lambdas=None, norms_out=None,
     return ws
 
 
+def dppf_distance_partials(x, sums_out, ws=None, d=None):
+    """Sums of squared distances to the column average over this column shard -> ``sums_out``
+    (fp64 CUDA tensor of M entries).  Returns the workspace used."""
+    M, d, ld = _dims(x, d)
+    if sums_out.dtype != torch.float64 or not sums_out.is_cuda or sums_out.numel() < M:
+        raise ValueError("sums_out must be an fp64 CUDA tensor with M entries")
+    ws = alloc_workspace(M, d, x.device) if ws is None else ws
+    _check(load().dppf_distance_partials(x.data_ptr(), M, d, ld, sums_out.data_ptr(), ws.data_ptr(), ws.numel(),
+                                         _stream()), "dppf_distance_partials")
+    return ws
+
+
+def dppf_update_from_sums(x, alpha, lam, sums, norms_out=None, d=None):
+    """Update pass on this column shard from the sums of squares totalled over all shards."""
+    M, d, ld = _dims(x, d)
+    if sums.dtype != torch.float64 or not sums.is_cuda or sums.numel() < M:
+        raise ValueError("sums must be an fp64 CUDA tensor with M entries")
+    _check(load().dppf_update_from_sums(x.data_ptr(), M, d, ld, alpha, lam, sums.data_ptr(), _ptr(norms_out),
+                                        _stream()), "dppf_update_from_sums")
+
+
 def debug_set_poll_limits(first_pass_polls=-1, later_pass_polls=-1) -> None:
     """Testing hook: poll budget of the bounded waits of later calls (negative = default)."""
     load().dppf_debug_set_poll_limits(int(first_pass_polls), int(later_pass_polls))
@@ -177,7 +211,7 @@ PUSH_FROM_AVERAGE, PUSH_FROM_CONSENSUS = 0, 1
 
 
 def dppf_consensus_general(x, alpha, lam, weights=None, push_from=PUSH_FROM_AVERAGE, two_term=False,
-                           norms_out=None, push_norms_out=None, ws=None, d=None):
+                           norms_out=None, push_norms_out=None, ws=None, d=None, path=PATH_AUTO):
     """General round in place on ``x[M, ld]``: consensus variable from ``weights`` (host
     sequence of M floats, None = plain average), push from x_A or x_C, optional second term."""
     M, d, ld = _dims(x, d)
@@ -187,9 +221,9 @@ def dppf_consensus_general(x, alpha, lam, weights=None, push_from=PUSH_FROM_AVER
         if len(weights) != M:
             raise ValueError("weights must have one entry per worker")
         wp = (ctypes.c_float * M)(*[float(v) for v in weights])
-    rc = load().dppf_consensus_general(x.data_ptr(), M, d, ld, alpha, lam, wp, int(push_from), int(bool(two_term)),
-                                       _ptr(norms_out), _ptr(push_norms_out), ws.data_ptr(), ws.numel(),
-                                       _stream())
+    rc = load().dppf_consensus_general_ex(x.data_ptr(), M, d, ld, alpha, lam, wp, int(push_from),
+                                          int(bool(two_term)), _ptr(norms_out), _ptr(push_norms_out),
+                                          ws.data_ptr(), ws.numel(), int(path), _stream())
     _check(rc, "dppf_consensus_general")
     return ws
 
@@ -241,12 +275,12 @@ def dppf_adamw_step(x, exp_avg, exp_avg_sq, g, lr, beta1, beta2, eps, weight_dec
 
 
 def dppf_adamw_step_and_consensus(x, exp_avg, exp_avg_sq, g, lr, beta1, beta2, eps, weight_decay, step,
-                                  alpha, lam, norms_out=None, ws=None, d=None):
+                                  alpha, lam, norms_out=None, ws=None, d=None, path=PATH_AUTO):
     M, d, ld = _same_shape(x, (exp_avg, exp_avg_sq, g), d)
     ws = alloc_workspace(M, d, x.device) if ws is None else ws
-    rc = load().dppf_adamw_step_and_consensus(
+    rc = load().dppf_adamw_step_and_consensus_ex(
         x.data_ptr(), exp_avg.data_ptr(), exp_avg_sq.data_ptr(), g.data_ptr(), M, d, ld, lr, beta1, beta2, eps,
-        weight_decay, int(step), alpha, lam, _ptr(norms_out), ws.data_ptr(), ws.numel(), _stream())
+        weight_decay, int(step), alpha, lam, _ptr(norms_out), ws.data_ptr(), ws.numel(), int(path), _stream())
     _check(rc, "dppf_adamw_step_and_consensus")
     return ws
 
@@ -293,3 +327,13 @@ def dppf_device_status(ws) -> int:
 
 def launch_count(M: int, d: int, path=PATH_AUTO, fused=False) -> int:
     return int(load().dppf_launch_count(int(M), int(d), int(path), int(bool(fused))))
+
+
+def adamw_launch_count(M: int, path=PATH_AUTO) -> int:
+    """Kernel launches of one dppf_adamw_step_and_consensus call."""
+    return int(load().dppf_launch_count(int(M), 1, int(path), 2))
+
+
+def dppf_static_device_status() -> int:
+    """Status word of the built-in scratch that dppf_consensus_static uses on the current device."""
+    return int(load().dppf_static_device_status(_stream()))

@@ -31,15 +31,23 @@ __device__ __forceinline__ void adamw4(float4 &x, float4 &m1, float4 &m2, float4
     adamw1(x.w, m1.w, m2.w, g.w, p);
 }
 
-// Distance pass with the AdamW step applied first; leaves the same partial sums and header
-// as distance_kernel, so update_kernel<M, false> completes the round.  Measured best with
-// the plain round's residency and two rows of loads in flight per thread.
+// Block shape of the kernels that fuse the AdamW step into the distance pass: four streams per
+// row (x, both moments, g) need more registers per thread than the plain round, so the blocks
+// are sized for 128 (M <= 8) or 255 (M > 8) registers and nothing spills.
 template <int M>
-__global__ void __launch_bounds__(Tuning<M>::kThreads, Tuning<M>::kBlocksPerSM)
-adamw_distance_kernel(const RoundArgs a, const AdamArgs p) {
-    constexpr int T = Tuning<M>::kThreads;
-    constexpr int G = 2;                               // rows whose loads are issued together
-    __shared__ double s_red[Tuning<M>::kWarps * M];
+struct AdamTuning {
+    static constexpr int kThreads = 256;
+    static constexpr int kBlocksPerSM = (M <= 8) ? 2 : 1;
+    static constexpr int kWarps = kThreads / 32;
+    static constexpr int kUnrollB = (M <= 4) ? 2 : 1;     // update pass: about 40-64 KB of loads in flight per SM
+};
+
+// Distance pass with the AdamW step applied first; leaves the same partial sums and header
+// as distance_kernel, so the ordinary update pass completes the round.  Loads of G rows are
+// issued together, ahead of their stores.
+template <int M, int G>
+__device__ __forceinline__ void adamw_distance_pass(const RoundArgs &a, const AdamArgs &p, double *s_red) {
+    constexpr int T = AdamTuning<M>::kThreads;
     const long long ntiles = (a.nvec + T - 1) / T;
     float acc[M];
 #pragma unroll
@@ -109,7 +117,7 @@ adamw_distance_kernel(const RoundArgs a, const AdamArgs p) {
     __syncthreads();
     if (threadIdx.x < M) {
         double sum = 0.0;
-        for (int w = 0; w < Tuning<M>::kWarps; ++w) sum += s_red[w * M + threadIdx.x];
+        for (int w = 0; w < AdamTuning<M>::kWarps; ++w) sum += s_red[w * M + threadIdx.x];
         a.partials[(long long)blockIdx.x * M + threadIdx.x] = sum;
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -118,6 +126,38 @@ adamw_distance_kernel(const RoundArgs a, const AdamArgs p) {
         a.hdr->grid = (int)gridDim.x;
         a.hdr->M = M;
     }
+}
+
+// Two-launch schedule (when a cooperative launch is refused, or on request): this kernel, then
+// adamw_update_kernel on the same grid.  On its own the pass needs a few more registers than
+// inside the persistent kernel, so its register budget is relaxed where that avoids spills.
+template <int M>
+__global__ void __launch_bounds__(AdamTuning<M>::kThreads, (M <= 6) ? AdamTuning<M>::kBlocksPerSM : 1)
+adamw_distance_kernel(const RoundArgs a, const AdamArgs p) {
+    __shared__ double s_red[AdamTuning<M>::kWarps * M];
+    adamw_distance_pass<M, (M == 16) ? 1 : 2>(a, p, s_red);
+}
+
+template <int M>
+__global__ void __launch_bounds__(AdamTuning<M>::kThreads, AdamTuning<M>::kBlocksPerSM)
+adamw_update_kernel(const RoundArgs a, int nblocks_a) {
+    __shared__ float s_c[M];
+    __shared__ int s_ok;
+    if (!finalise(a, M, nblocks_a, s_c, &s_ok)) return;
+    update_pass<M, AdamTuning<M>::kUnrollB, AdamTuning<M>::kThreads>(a, s_c);
+}
+
+// One persistent cooperative launch: AdamW step + distance pass, grid barrier, update pass.
+template <int M>
+__global__ void __launch_bounds__(AdamTuning<M>::kThreads, AdamTuning<M>::kBlocksPerSM)
+adamw_round_kernel(const RoundArgs a, const AdamArgs p) {
+    __shared__ double s_red[AdamTuning<M>::kWarps * M];
+    __shared__ float s_c[M];
+    __shared__ int s_ok;
+    adamw_distance_pass<M, 2>(a, p, s_red);
+    cg::this_grid().sync();
+    if (!finalise(a, M, (int)gridDim.x, s_c, &s_ok)) return;
+    update_pass<M, AdamTuning<M>::kUnrollB, AdamTuning<M>::kThreads>(a, s_c);
 }
 
 __global__ void __launch_bounds__(kThreads) adamw_step_kernel(float *x, const AdamArgs p, long long d, long long ld,

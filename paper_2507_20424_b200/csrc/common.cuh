@@ -39,6 +39,7 @@ struct RoundArgs {
     WsHeader *hdr;
     double *partials; // [grid, M]
     int M;            // runtime copy (generic kernels)
+    int spin_first, spin_later;   // staged kernel: mbarrier polls before a wait gives up (distance / update pass)
 };
 
 // ---------------------------------------------------------------- memory access helpers

@@ -3,7 +3,8 @@
 //   common.cuh          constants, argument structs, cache-hinted accesses, rounded arithmetic
 //   round_register.cuh  register-resident round kernels (two-launch and cooperative schedules)
 //   adamw.cuh           AdamW local step, stand-alone and fused into the distance pass
-//   round_staged.cuh    staged persistent round kernel (bulk async copies into a shared-memory ring)
+//   chunk_ring.cuh      shared-memory chunk ring of the staged kernels (bulk async copies, bounded waits)
+//   round_staged.cuh    staged persistent round kernel, one round per launch
 //   round_multi.cuh     several rounds in one launch (update pass of round k + distances of round k+1)
 //   round_general.cuh   general round (weighted consensus variable, push reference, two-term push)
 //   round_generic.cuh   any worker count up to 1024, stand-alone SGD-momentum local step
@@ -33,6 +34,7 @@
 #include "common.cuh"
 #include "round_register.cuh"
 #include "adamw.cuh"
+#include "chunk_ring.cuh"
 #include "round_staged.cuh"
 #include "round_multi.cuh"
 #include "round_general.cuh"
@@ -66,6 +68,10 @@ bool coop_supported(int dev) {
     return c != 0;
 }
 
+// Poll limits of the bounded waits of the staged kernels (distance pass / later passes).  Only
+// the testing hook dppf_debug_set_poll_limits changes them.
+std::atomic<int> g_spin_first{kSpinLimit}, g_spin_later{kSpinLimit};
+
 int max_blocks_for(int M) { return M <= kMaxTemplateM ? kMaxBlocksSmallM : kMaxBlocksLargeM; }
 
 size_t norms_stage_offset(int M) {
@@ -81,6 +87,12 @@ bool finite_all(std::initializer_list<float> vals) {
     for (float f : vals)
         if (!std::isfinite(f)) return false;
     return true;
+}
+
+// Bytes from the first element of row 0 to the last element of row M-1 (a column shard of a
+// wider buffer ends before its last row's stride does).
+size_t extent_bytes(int M, int64_t d, int64_t ld) {
+    return ((size_t)(M - 1) * (size_t)ld + (size_t)d) * sizeof(float);
 }
 
 bool aligned128(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 127u) == 0; }
@@ -112,8 +124,21 @@ int blocks_per_sm(K kernel, int dev, int M, int kind, int threads, size_t dyn_sm
 }
 
 template <int M>
+int launch_rounds_m(RoundsArgs &a, int path, int dev, cudaStream_t s, bool *refused);
+RoundsArgs one_round_args(const RoundArgs &a);
+
+template <int M>
 int launch_round_m(RoundArgs a, bool fused, int path, int dev, cudaStream_t s) {
-    if (path == DPPF_PATH_STAGED && !fused && coop_supported(dev)) {
+    if (path == DPPF_PATH_STAGED && !fused && M > 8) {
+        // above eight rows the multi-round kernel (row copies issued by one lane each) is the faster
+        // staged kernel; a single round is its two-pass special case
+        RoundsArgs ra = one_round_args(a);
+        bool refused = false;
+        const int rc = launch_rounds_m<M>(ra, DPPF_PATH_STAGED, dev, s, &refused);
+        if (rc == DPPF_OK || !refused) return rc;
+        path = DPPF_PATH_TWO_KERNEL;
+    }
+    if constexpr (M <= 8) if (path == DPPF_PATH_STAGED && !fused && coop_supported(dev)) {
         constexpr size_t smem = StagedShape<M>::kSmemBytes;
         if (g_occ[dev][M][2].load(std::memory_order_relaxed) == 0 &&
             cudaFuncSetAttribute(round_kernel_staged<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
@@ -219,8 +244,8 @@ int launch_local_step(float *x, float *v, const float *g, int M, int64_t d, int6
 int resolve_path(int path, int M, bool fused) {
     if (M > kMaxTemplateM) return DPPF_PATH_TWO_KERNEL;
     if (fused && path == DPPF_PATH_STAGED) return DPPF_PATH_COOPERATIVE;   // no staged kernel with the local step
-    // one launch per round; staging through shared memory pays off up to eight rows
-    if (path == DPPF_PATH_AUTO) return (fused || M > 8) ? DPPF_PATH_COOPERATIVE : DPPF_PATH_STAGED;
+    // one launch per round, rows staged through shared memory
+    if (path == DPPF_PATH_AUTO) return fused ? DPPF_PATH_COOPERATIVE : DPPF_PATH_STAGED;
     return path;
 }
 
@@ -233,7 +258,7 @@ int run_round(float *x, float *v, const float *g, int M, int64_t d, int64_t ld, 
         path != DPPF_PATH_STAGED)
         return DPPF_ERR_INVALID_ARG;
     if (!finite_all({alpha, lambda})) return DPPF_ERR_INVALID_ARG;
-    const size_t bytes = (size_t)M * (size_t)ld * sizeof(float);
+    const size_t bytes = extent_bytes(M, d, ld);
     if (fused) {
         if ((rc = check_layout(v, M, d, ld)) != DPPF_OK) return rc;
         if ((rc = check_layout(g, M, d, ld)) != DPPF_OK) return rc;
@@ -257,6 +282,8 @@ int run_round(float *x, float *v, const float *g, int M, int64_t d, int64_t ld, 
     a.partials = reinterpret_cast<double *>(static_cast<unsigned char *>(ws) + kHeaderBytes);
     a.norms_stage = reinterpret_cast<float *>(static_cast<unsigned char *>(ws) + norms_stage_offset(M));
     a.M = M;
+    a.spin_first = g_spin_first.load(std::memory_order_relaxed);
+    a.spin_later = g_spin_later.load(std::memory_order_relaxed);
 
     if (M == 1) {   // x_A == x_1: distance 0, replica unchanged
         if (fused && (rc = launch_local_step(x, v, g, M, d, ld, lr, mu, wd, dev, s)) != DPPF_OK) return rc;
@@ -272,6 +299,82 @@ int run_round(float *x, float *v, const float *g, int M, int64_t d, int64_t ld, 
 #undef DPPF_CASE
         default: return launch_round_generic(a, fused, dev, s);
     }
+}
+
+// ---------------------------------------------------------------- the two passes as separate calls
+template <int M>
+int distance_only_m(const RoundArgs &a, int dev, cudaStream_t s) {
+    constexpr int T = Tuning<M>::kThreads;
+    const int sms = sm_count(dev);
+    if (sms <= 0) return -1;
+    const long long tile_vecs = (long long)T * Tuning<M>::kUnrollA;
+    long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
+    if (ntiles < 1) ntiles = 1;
+    long long grid = (long long)sms * Tuning<M>::kBlocksPerSM;
+    if (grid > ntiles) grid = ntiles;
+    if (grid > kMaxBlocksSmallM) grid = kMaxBlocksSmallM;
+    distance_kernel<M, false><<<(unsigned)grid, T, 0, s>>>(a);
+    return cudaGetLastError() == cudaSuccess ? (int)grid : -1;
+}
+
+// Distance pass alone; returns the number of blocks that wrote partial sums, -1 on failure.
+int launch_distance_only(const RoundArgs &a, int M, int dev, cudaStream_t s) {
+    switch (M) {
+#define DPPF_CASE(MM) case MM: return distance_only_m<MM>(a, dev, s);
+        DPPF_CASE(1) DPPF_CASE(2) DPPF_CASE(3) DPPF_CASE(4) DPPF_CASE(5) DPPF_CASE(6) DPPF_CASE(7) DPPF_CASE(8)
+        DPPF_CASE(9) DPPF_CASE(10) DPPF_CASE(11) DPPF_CASE(12) DPPF_CASE(13) DPPF_CASE(14) DPPF_CASE(15)
+        DPPF_CASE(16)
+#undef DPPF_CASE
+        default: break;
+    }
+    const int sms = sm_count(dev);
+    if (sms <= 0) return -1;
+    long long ntiles = (a.nvec + kThreads - 1) / kThreads;
+    if (ntiles < 1) ntiles = 1;
+    long long grid = (long long)sms * 2;
+    if (grid > ntiles) grid = ntiles;
+    if (grid > kMaxBlocksLargeM) grid = kMaxBlocksLargeM;
+    const size_t smem_a = (size_t)kWarps * a.M * sizeof(float);
+    if (smem_a > 48 * 1024 &&
+        cudaFuncSetAttribute(distance_kernel_generic<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)smem_a) != cudaSuccess)
+        return -1;
+    distance_kernel_generic<false><<<(unsigned)grid, kThreads, smem_a, s>>>(a);
+    return cudaGetLastError() == cudaSuccess ? (int)grid : -1;
+}
+
+template <int M>
+int update_only_m(const RoundArgs &a, int dev, cudaStream_t s) {
+    constexpr int T = Tuning<M>::kThreads;
+    const int sms = sm_count(dev);
+    if (sms <= 0) return DPPF_ERR_CUDA;
+    const long long tile_vecs = (long long)T * Tuning<M>::kUnrollB;
+    long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
+    if (ntiles < 1) ntiles = 1;
+    long long grid = (long long)sms * Tuning<M>::kBlocksPerSM;
+    if (grid > ntiles) grid = ntiles;
+    update_kernel<M, false><<<(unsigned)grid, T, 0, s>>>(a, 1);
+    return cudaGetLastError() == cudaSuccess ? DPPF_OK : DPPF_ERR_CUDA;
+}
+
+// Update pass alone, from M caller-provided sums of squares (a.partials, a.hdr == nullptr).
+int launch_update_only(const RoundArgs &a, int M, int dev, cudaStream_t s) {
+    switch (M) {
+#define DPPF_CASE(MM) case MM: return update_only_m<MM>(a, dev, s);
+        DPPF_CASE(1) DPPF_CASE(2) DPPF_CASE(3) DPPF_CASE(4) DPPF_CASE(5) DPPF_CASE(6) DPPF_CASE(7) DPPF_CASE(8)
+        DPPF_CASE(9) DPPF_CASE(10) DPPF_CASE(11) DPPF_CASE(12) DPPF_CASE(13) DPPF_CASE(14) DPPF_CASE(15)
+        DPPF_CASE(16)
+#undef DPPF_CASE
+        default: break;
+    }
+    const int sms = sm_count(dev);
+    if (sms <= 0) return DPPF_ERR_CUDA;
+    long long ntiles = (a.nvec + kThreads - 1) / kThreads;
+    if (ntiles < 1) ntiles = 1;
+    long long grid = (long long)sms * 2;
+    if (grid > ntiles) grid = ntiles;
+    update_kernel_generic<<<(unsigned)grid, kThreads, (size_t)a.M * sizeof(float), s>>>(a, 1);
+    return cudaGetLastError() == cudaSuccess ? DPPF_OK : DPPF_ERR_CUDA;
 }
 
 // ---------------------------------------------------------------- built-in scratch
@@ -302,10 +405,23 @@ int static_ws_address(int dev, void **out) {
 
 
 // ---------------------------------------------------------------- several rounds per launch: host side
-// Poll limits of the bounded waits (first pass / later passes).  Only the testing hook
-// dppf_debug_set_poll_limits changes them.
-std::atomic<int> g_spin_first{kSpinLimit}, g_spin_later{kSpinLimit};
 std::atomic<int> g_rounds_ready[64][kMaxTemplateM + 1][2];   // [][][0] staged, [1] register: blocks per SM
+
+RoundsArgs one_round_args(const RoundArgs &a) {
+    RoundsArgs r;
+    r.x = a.x; r.d = a.d; r.ld = a.ld; r.nvec = a.nvec;
+    r.alpha = a.alpha;
+    r.n_rounds = 1;
+    r.spin_first = a.spin_first;
+    r.spin_later = a.spin_later;
+    r.norms_all = a.norms_out;
+    r.norms_stage = a.norms_stage;
+    r.hdr = a.hdr;
+    r.partials = a.partials;
+    r.partials_half = (long long)(kMaxBlocksSmallM / 2) * a.M;
+    r.lambdas[0] = a.lambda;
+    return r;
+}
 
 // One launch of up to kMaxRoundsPerLaunch rounds.  DPPF_ERR_CUDA + *refused = true when the
 // runtime will not launch cooperatively (caller falls back to single rounds).
@@ -383,35 +499,45 @@ int launch_rounds(RoundsArgs &a, int M, int path, int dev, cudaStream_t s, bool 
 std::atomic<int> g_general_ready[64][kMaxTemplateM + 1];
 
 template <int M>
-int launch_general_m(const GeneralArgs &a, int dev, cudaStream_t s) {
-    if (!coop_supported(dev)) return DPPF_ERR_CUDA;
-    constexpr size_t smem = StagedShape<M>::kSmemBytes;
-    if (g_general_ready[dev][M].load(std::memory_order_relaxed) == 0) {
-        if (cudaFuncSetAttribute(general_round_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-            cudaSuccess) {
-            cudaGetLastError();
-            return DPPF_ERR_CUDA;
-        }
-        int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, general_round_kernel<M>, kGeneralThreads, smem) !=
-                cudaSuccess || n < 1)
-            return DPPF_ERR_CUDA;
-        g_general_ready[dev][M].store(1, std::memory_order_relaxed);
-    }
+int launch_general_m(const GeneralArgs &a, int path, int dev, cudaStream_t s) {
     const int sms = sm_count(dev);
     if (sms <= 0) return DPPF_ERR_CUDA;
-    const long long nchunks = (a.nvec * 4 + StagedShape<M>::kChunk - 1) / StagedShape<M>::kChunk;
-    long long grid = sms;
-    if (grid > nchunks) grid = nchunks;
-    if (grid < 1) grid = 1;
     GeneralArgs args = a;
-    void *params[] = {&args};
-    if (cudaLaunchCooperativeKernel((const void *)general_round_kernel<M>, dim3((unsigned)grid),
-                                    dim3(kGeneralThreads), params, smem, s) != cudaSuccess) {
-        cudaGetLastError();
-        return DPPF_ERR_CUDA;
+    if (path != DPPF_PATH_TWO_KERNEL && coop_supported(dev)) {
+        constexpr size_t smem = StagedShape<M>::kSmemBytes;
+        bool ready = g_general_ready[dev][M].load(std::memory_order_relaxed) != 0;
+        if (!ready) {
+            int n = 0;
+            ready = cudaFuncSetAttribute(general_round_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem) == cudaSuccess &&
+                    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, general_round_kernel<M>, kGeneralThreads,
+                                                                  smem) == cudaSuccess && n >= 1;
+            if (ready) g_general_ready[dev][M].store(1, std::memory_order_relaxed);
+            else cudaGetLastError();
+        }
+        if (ready) {
+            const long long nchunks = (a.nvec * 4 + StagedShape<M>::kChunk - 1) / StagedShape<M>::kChunk;
+            long long grid = sms;
+            if (grid > nchunks) grid = nchunks;
+            if (grid > kMaxBlocksSmallM / 2) grid = kMaxBlocksSmallM / 2;
+            if (grid < 1) grid = 1;
+            void *params[] = {&args};
+            if (cudaLaunchCooperativeKernel((const void *)general_round_kernel<M>, dim3((unsigned)grid),
+                                            dim3(kGeneralThreads), params, smem, s) == cudaSuccess)
+                return DPPF_OK;
+            cudaGetLastError();                         // refused (blocks cannot all be resident now): two launches
+        }
     }
-    return DPPF_OK;
+    constexpr int T = Tuning<M>::kThreads;
+    long long ntiles = (a.nvec + T - 1) / T;
+    if (ntiles < 1) ntiles = 1;
+    long long grid = (long long)sms * Tuning<M>::kBlocksPerSM;
+    if (grid > ntiles) grid = ntiles;
+    if (grid > kMaxBlocksSmallM / 2) grid = kMaxBlocksSmallM / 2;   // the partials hold 2M sums per block
+    args.grid_a = (int)grid;
+    general_distance_kernel<M><<<(unsigned)grid, T, 0, s>>>(args);
+    general_update_kernel<M><<<(unsigned)grid, T, 0, s>>>(args);
+    return cudaGetLastError() == cudaSuccess ? DPPF_OK : DPPF_ERR_CUDA;
 }
 
 
@@ -439,7 +565,7 @@ int check_adam_buffers(const float *x, const float *m1, const float *m2, const f
     if ((rc = check_layout(m1, M, d, ld)) != DPPF_OK) return rc;
     if ((rc = check_layout(m2, M, d, ld)) != DPPF_OK) return rc;
     if ((rc = check_layout(g, M, d, ld)) != DPPF_OK) return rc;
-    const size_t bytes = (size_t)M * (size_t)ld * sizeof(float);
+    const size_t bytes = extent_bytes(M, d, ld);
     const void *bufs[4] = {x, m1, m2, g};
     for (int i = 0; i < 4; ++i)
         for (int j = i + 1; j < 4; ++j)
@@ -459,19 +585,40 @@ int launch_adamw_step(float *x, const AdamArgs &p, int M, int64_t d, int64_t ld,
     return cudaGetLastError() == cudaSuccess ? DPPF_OK : DPPF_ERR_CUDA;
 }
 
+std::atomic<int> g_adamw_occ[64][kMaxTemplateM + 1];
+
 template <int M>
-int launch_adamw_round_m(const RoundArgs &a, const AdamArgs &p, int dev, cudaStream_t s) {
-    constexpr int T = Tuning<M>::kThreads;
+int launch_adamw_round_m(const RoundArgs &a, const AdamArgs &p, int path, int dev, cudaStream_t s) {
+    constexpr int T = AdamTuning<M>::kThreads;
     const int sms = sm_count(dev);
     if (sms <= 0) return DPPF_ERR_CUDA;
-    const long long tile_vecs = (long long)T * Tuning<M>::kUnrollB;
+    int per_sm = g_adamw_occ[dev][M].load(std::memory_order_relaxed);
+    if (per_sm == 0) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, adamw_round_kernel<M>, T, 0) != cudaSuccess ||
+            per_sm < 1) {
+            cudaGetLastError();
+            return DPPF_ERR_CUDA;
+        }
+        g_adamw_occ[dev][M].store(per_sm, std::memory_order_relaxed);
+    }
+    if (per_sm > AdamTuning<M>::kBlocksPerSM) per_sm = AdamTuning<M>::kBlocksPerSM;
+    const long long tile_vecs = (long long)T * AdamTuning<M>::kUnrollB;
     long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
     if (ntiles < 1) ntiles = 1;
-    long long grid = (long long)sms * Tuning<M>::kBlocksPerSM;
+    long long grid = (long long)sms * per_sm;            // the same grid for both schedules: same partial sums
     if (grid > ntiles) grid = ntiles;
     if (grid > kMaxBlocksSmallM) grid = kMaxBlocksSmallM;
+    if (path != DPPF_PATH_TWO_KERNEL && coop_supported(dev)) {
+        RoundArgs aa = a;
+        AdamArgs pp = p;
+        void *params[] = {&aa, &pp};
+        if (cudaLaunchCooperativeKernel((const void *)adamw_round_kernel<M>, dim3((unsigned)grid), dim3(T), params, 0,
+                                        s) == cudaSuccess)
+            return DPPF_OK;
+        cudaGetLastError();                              // refused: two plain launches
+    }
     adamw_distance_kernel<M><<<(unsigned)grid, T, 0, s>>>(a, p);
-    update_kernel<M, false><<<(unsigned)grid, T, 0, s>>>(a, (int)grid);
+    adamw_update_kernel<M><<<(unsigned)grid, T, 0, s>>>(a, (int)grid);
     return cudaGetLastError() == cudaSuccess ? DPPF_OK : DPPF_ERR_CUDA;
 }
 
@@ -504,7 +651,7 @@ int dppf_local_step(float *x, float *v, const float *g, int M, int64_t d, int64_
     if ((rc = check_layout(v, M, d, ld)) != DPPF_OK) return rc;
     if ((rc = check_layout(g, M, d, ld)) != DPPF_OK) return rc;
     if (!finite_all({lr, momentum, weight_decay})) return DPPF_ERR_INVALID_ARG;
-    const size_t bytes = (size_t)M * (size_t)ld * sizeof(float);
+    const size_t bytes = extent_bytes(M, d, ld);
     if (overlap(x, bytes, v, bytes) || overlap(x, bytes, g, bytes) || overlap(v, bytes, g, bytes)) return DPPF_ERR_INVALID_ARG;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DPPF_ERR_CUDA;
@@ -576,7 +723,66 @@ const char *dppf_status_string(int status) {
 int dppf_launch_count(int M, int64_t d, int path, int fused) {
     if (M < 1 || M > DPPF_MAX_WORKERS || d < 1) return 0;
     if (M == 1) return fused ? 2 : 1;                       // [local step], zero norms
+    if (fused == 2) return (M > kMaxTemplateM) ? 0 : (path == DPPF_PATH_TWO_KERNEL ? 2 : 1);   // AdamW fused
     return resolve_path(path, M, fused != 0) == DPPF_PATH_TWO_KERNEL ? 2 : 1;
+}
+
+// ---- a round split at its reduction (column shards of the replicas on several GPUs)
+
+int dppf_distance_partials(const float *x, int M, int64_t d, int64_t ld, double *sums_out, void *ws,
+                           size_t ws_bytes, void *cuda_stream) {
+    int rc = check_layout(x, M, d, ld);
+    if (rc != DPPF_OK) return rc;
+    if (!sums_out || (reinterpret_cast<uintptr_t>(sums_out) & 7u)) return DPPF_ERR_INVALID_ARG;
+    if (!ws) return DPPF_ERR_INVALID_ARG;
+    if (!aligned128(ws)) return DPPF_ERR_ALIGNMENT;
+    if (ws_bytes < workspace_bytes(M)) return DPPF_ERR_WORKSPACE;
+    const size_t bytes = extent_bytes(M, d, ld);
+    if (overlap(x, bytes, ws, workspace_bytes(M)) || overlap(x, bytes, sums_out, (size_t)M * sizeof(double)) ||
+        overlap(ws, workspace_bytes(M), sums_out, (size_t)M * sizeof(double)))
+        return DPPF_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DPPF_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    RoundArgs a;
+    a.x = const_cast<float *>(x); a.v = nullptr; a.g = nullptr;     // the distance pass only reads x
+    a.d = d; a.ld = ld; a.nvec = d / 4;
+    a.alpha = 0.f; a.lambda = 0.f; a.lr = a.mu = a.wd = 0.f;
+    a.norms_out = nullptr;
+    a.hdr = reinterpret_cast<WsHeader *>(ws);
+    a.partials = reinterpret_cast<double *>(static_cast<unsigned char *>(ws) + kHeaderBytes);
+    a.norms_stage = reinterpret_cast<float *>(static_cast<unsigned char *>(ws) + norms_stage_offset(M));
+    a.M = M;
+    a.spin_first = a.spin_later = kSpinLimit;
+    const int grid = launch_distance_only(a, M, dev, s);
+    if (grid <= 0) return DPPF_ERR_CUDA;
+    const int warps = M < 16 ? M : 16;
+    sum_partials_kernel<<<1, 32 * warps, 0, s>>>(a.partials, grid, M, sums_out);
+    return cudaGetLastError() == cudaSuccess ? DPPF_OK : DPPF_ERR_CUDA;
+}
+
+int dppf_update_from_sums(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda, const double *sums,
+                          float *norms_out, void *cuda_stream) {
+    int rc = check_layout(x, M, d, ld);
+    if (rc != DPPF_OK) return rc;
+    if (!sums || (reinterpret_cast<uintptr_t>(sums) & 7u)) return DPPF_ERR_INVALID_ARG;
+    if (!finite_all({alpha, lambda})) return DPPF_ERR_INVALID_ARG;
+    const size_t bytes = extent_bytes(M, d, ld);
+    if (overlap(x, bytes, sums, (size_t)M * sizeof(double))) return DPPF_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DPPF_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    RoundArgs a;
+    a.x = x; a.v = nullptr; a.g = nullptr;
+    a.d = d; a.ld = ld; a.nvec = d / 4;
+    a.alpha = alpha; a.lambda = lambda; a.lr = a.mu = a.wd = 0.f;
+    a.norms_out = norms_out;
+    a.hdr = nullptr;                                   // the sums are the caller's: no header, no staging
+    a.partials = const_cast<double *>(sums);
+    a.norms_stage = nullptr;
+    a.M = M;
+    a.spin_first = a.spin_later = kSpinLimit;
+    return launch_update_only(a, M, dev, s);
 }
 
 int dppf_consensus_rounds_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
@@ -598,14 +804,14 @@ int dppf_consensus_rounds_ex(float *x, int M, int64_t d, int64_t ld, float alpha
     if (!ws) return DPPF_ERR_INVALID_ARG;
     if (!aligned128(ws)) return DPPF_ERR_ALIGNMENT;
     if (ws_bytes < workspace_bytes(M)) return DPPF_ERR_WORKSPACE;
-    const size_t bytes = (size_t)M * (size_t)ld * sizeof(float);
+    const size_t bytes = extent_bytes(M, d, ld);
     if (overlap(x, bytes, ws, workspace_bytes(M))) return DPPF_ERR_INVALID_ARG;
     if (norms_out && overlap(x, bytes, norms_out, (size_t)n_rounds * M * sizeof(float))) return DPPF_ERR_INVALID_ARG;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DPPF_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
 
-    if (path == DPPF_PATH_AUTO) path = (M <= 8) ? DPPF_PATH_STAGED : DPPF_PATH_COOPERATIVE;
+    if (path == DPPF_PATH_AUTO) path = DPPF_PATH_STAGED;
     bool single_rounds = (M == 1 || M > kMaxTemplateM || path == DPPF_PATH_TWO_KERNEL);
     int done = 0;
     while (!single_rounds && done < n_rounds) {
@@ -656,6 +862,7 @@ int dppf_consensus_static(float *x, int M, int64_t d, int64_t ld, float alpha, f
     if (workspace_bytes(M) > kStaticWsBytes) return DPPF_ERR_WORKSPACE;
     int rc = check_layout(x, M, d, ld);      // reject bad arguments before any CUDA call
     if (rc != DPPF_OK) return rc;
+    if (!finite_all({alpha, lambda})) return DPPF_ERR_INVALID_ARG;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DPPF_ERR_CUDA;
     void *ws = nullptr;
@@ -664,24 +871,36 @@ int dppf_consensus_static(float *x, int M, int64_t d, int64_t ld, float alpha, f
                      DPPF_PATH_AUTO, false, static_cast<cudaStream_t>(cuda_stream));
 }
 
-int dppf_consensus_general(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda, const float *weights_host,
-                           int push_from, int two_term, float *norms_out, float *push_norms_out, void *ws,
-                           size_t ws_bytes, void *cuda_stream) {
+int dppf_static_device_status(void *cuda_stream) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DPPF_ERR_CUDA;
+    void *ws = nullptr;
+    const int rc = static_ws_address(dev, &ws);
+    if (rc != DPPF_OK) return rc;
+    return dppf_device_status(ws, cuda_stream);
+}
+
+int dppf_consensus_general_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
+                              const float *weights_host, int push_from, int two_term, float *norms_out,
+                              float *push_norms_out, void *ws, size_t ws_bytes, int path, void *cuda_stream) {
     int rc = check_layout(x, M, d, ld);
     if (rc != DPPF_OK) return rc;
     if (M > kMaxTemplateM) return DPPF_ERR_INVALID_ARG;
+    if (path != DPPF_PATH_AUTO && path != DPPF_PATH_TWO_KERNEL && path != DPPF_PATH_STAGED) return DPPF_ERR_INVALID_ARG;
     if (push_from != DPPF_PUSH_FROM_AVERAGE && push_from != DPPF_PUSH_FROM_CONSENSUS) return DPPF_ERR_INVALID_ARG;
     if (!finite_all({alpha, lambda})) return DPPF_ERR_INVALID_ARG;
     if (!ws) return DPPF_ERR_INVALID_ARG;
     if (!aligned128(ws)) return DPPF_ERR_ALIGNMENT;
     if (ws_bytes < workspace_bytes(M)) return DPPF_ERR_WORKSPACE;
-    const size_t bytes = (size_t)M * (size_t)ld * sizeof(float);
+    const size_t bytes = extent_bytes(M, d, ld);
     if (overlap(x, bytes, ws, workspace_bytes(M))) return DPPF_ERR_INVALID_ARG;
     GeneralArgs a;
     double wsum = 0.0;
+    bool uniform = true;
     for (int m = 0; m < M; ++m) {
         const float w = weights_host ? weights_host[m] : 1.0f;
         if (!std::isfinite(w)) return DPPF_ERR_INVALID_ARG;
+        if (weights_host && w != weights_host[0]) uniform = false;
         wsum += (double)w;
     }
     if (!(wsum != 0.0) || !std::isfinite(wsum)) return DPPF_ERR_INVALID_ARG;
@@ -693,18 +912,29 @@ int dppf_consensus_general(float *x, int M, int64_t d, int64_t ld, float alpha, 
     a.alpha = alpha; a.lambda = lambda;
     a.push_from_c = (push_from == DPPF_PUSH_FROM_CONSENSUS) ? 1 : 0;
     a.two_term = two_term ? 1 : 0;
+    a.uniform = uniform ? 1 : 0;
+    a.spin_first = g_spin_first.load(std::memory_order_relaxed);
+    a.spin_later = g_spin_later.load(std::memory_order_relaxed);
+    a.grid_a = 0;
     a.norms_out = norms_out; a.push_norms_out = push_norms_out;
     a.hdr = reinterpret_cast<WsHeader *>(ws);
     a.partials = reinterpret_cast<double *>(static_cast<unsigned char *>(ws) + kHeaderBytes);
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     switch (M) {
-#define DPPF_CASE(MM) case MM: return launch_general_m<MM>(a, dev, s);
+#define DPPF_CASE(MM) case MM: return launch_general_m<MM>(a, path, dev, s);
         DPPF_CASE(1) DPPF_CASE(2) DPPF_CASE(3) DPPF_CASE(4) DPPF_CASE(5) DPPF_CASE(6) DPPF_CASE(7) DPPF_CASE(8)
         DPPF_CASE(9) DPPF_CASE(10) DPPF_CASE(11) DPPF_CASE(12) DPPF_CASE(13) DPPF_CASE(14) DPPF_CASE(15)
         DPPF_CASE(16)
 #undef DPPF_CASE
         default: return DPPF_ERR_INVALID_ARG;
     }
+}
+
+int dppf_consensus_general(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda, const float *weights_host,
+                           int push_from, int two_term, float *norms_out, float *push_norms_out, void *ws,
+                           size_t ws_bytes, void *cuda_stream) {
+    return dppf_consensus_general_ex(x, M, d, ld, alpha, lambda, weights_host, push_from, two_term, norms_out,
+                                     push_norms_out, ws, ws_bytes, DPPF_PATH_AUTO, cuda_stream);
 }
 
 int dppf_adamw_step(float *x, float *exp_avg, float *exp_avg_sq, const float *g, int M, int64_t d, int64_t ld,
@@ -718,20 +948,21 @@ int dppf_adamw_step(float *x, float *exp_avg, float *exp_avg_sq, const float *g,
     return launch_adamw_step(x, p, M, d, ld, dev, static_cast<cudaStream_t>(cuda_stream));
 }
 
-int dppf_adamw_step_and_consensus(float *x, float *exp_avg, float *exp_avg_sq, const float *g, int M, int64_t d,
-                                  int64_t ld, float lr, float beta1, float beta2, float eps, float weight_decay,
-                                  int step, float alpha, float lambda, float *norms_out, void *ws, size_t ws_bytes,
-                                  void *cuda_stream) {
+int dppf_adamw_step_and_consensus_ex(float *x, float *exp_avg, float *exp_avg_sq, const float *g, int M, int64_t d,
+                                     int64_t ld, float lr, float beta1, float beta2, float eps, float weight_decay,
+                                     int step, float alpha, float lambda, float *norms_out, void *ws,
+                                     size_t ws_bytes, int path, void *cuda_stream) {
     int rc = check_adam_buffers(x, exp_avg, exp_avg_sq, g, M, d, ld);
     if (rc != DPPF_OK) return rc;
     if (M > kMaxTemplateM) return DPPF_ERR_INVALID_ARG;
+    if (path != DPPF_PATH_AUTO && path != DPPF_PATH_TWO_KERNEL && path != DPPF_PATH_COOPERATIVE) return DPPF_ERR_INVALID_ARG;
     if (!finite_all({alpha, lambda})) return DPPF_ERR_INVALID_ARG;
     AdamArgs p;
     if ((rc = make_adam_args(exp_avg, exp_avg_sq, g, lr, beta1, beta2, eps, weight_decay, step, &p)) != DPPF_OK) return rc;
     if (!ws) return DPPF_ERR_INVALID_ARG;
     if (!aligned128(ws)) return DPPF_ERR_ALIGNMENT;
     if (ws_bytes < workspace_bytes(M)) return DPPF_ERR_WORKSPACE;
-    const size_t bytes = (size_t)M * (size_t)ld * sizeof(float);
+    const size_t bytes = extent_bytes(M, d, ld);
     if (overlap(x, bytes, ws, workspace_bytes(M))) return DPPF_ERR_INVALID_ARG;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DPPF_ERR_CUDA;
@@ -745,19 +976,28 @@ int dppf_adamw_step_and_consensus(float *x, float *exp_avg, float *exp_avg_sq, c
     a.partials = reinterpret_cast<double *>(static_cast<unsigned char *>(ws) + kHeaderBytes);
     a.norms_stage = reinterpret_cast<float *>(static_cast<unsigned char *>(ws) + norms_stage_offset(M));
     a.M = M;
+    a.spin_first = a.spin_later = kSpinLimit;
     if (M == 1) {
         if ((rc = launch_adamw_step(x, p, M, d, ld, dev, s)) != DPPF_OK) return rc;
         zero_norms_kernel<<<1, 32, 0, s>>>(norms_out, a.norms_stage, a.hdr);
         return cudaGetLastError() == cudaSuccess ? DPPF_OK : DPPF_ERR_CUDA;
     }
     switch (M) {
-#define DPPF_CASE(MM) case MM: return launch_adamw_round_m<MM>(a, p, dev, s);
+#define DPPF_CASE(MM) case MM: return launch_adamw_round_m<MM>(a, p, path, dev, s);
         DPPF_CASE(2) DPPF_CASE(3) DPPF_CASE(4) DPPF_CASE(5) DPPF_CASE(6) DPPF_CASE(7) DPPF_CASE(8)
         DPPF_CASE(9) DPPF_CASE(10) DPPF_CASE(11) DPPF_CASE(12) DPPF_CASE(13) DPPF_CASE(14) DPPF_CASE(15)
         DPPF_CASE(16)
 #undef DPPF_CASE
         default: return DPPF_ERR_INVALID_ARG;
     }
+}
+
+int dppf_adamw_step_and_consensus(float *x, float *exp_avg, float *exp_avg_sq, const float *g, int M, int64_t d,
+                                  int64_t ld, float lr, float beta1, float beta2, float eps, float weight_decay,
+                                  int step, float alpha, float lambda, float *norms_out, void *ws, size_t ws_bytes,
+                                  void *cuda_stream) {
+    return dppf_adamw_step_and_consensus_ex(x, exp_avg, exp_avg_sq, g, M, d, ld, lr, beta1, beta2, eps, weight_decay,
+                                            step, alpha, lambda, norms_out, ws, ws_bytes, DPPF_PATH_AUTO, cuda_stream);
 }
 
 // ---- host-side scalars of a run (no device work)

@@ -1,6 +1,7 @@
 // General round (arbitrary consensus variable, push from x_A or x_C, two-term push) on the staged pipeline.
 #pragma once
-#include "round_staged.cuh"
+#include "round_register.cuh"
+#include "chunk_ring.cuh"
 
 namespace {
 
@@ -24,10 +25,13 @@ struct GeneralArgs {
     float alpha, lambda;
     float wn[kMaxTemplateM];     // w_m / sum w
     int push_from_c, two_term;
+    int uniform;                 // all weights equal: x_C is x_A, bit for bit
+    int spin_first, spin_later;  // mbarrier polls before a wait gives up (distance / update pass)
     float *norms_out;            // ||x_m - x_A|| before the round, may be null
     float *push_norms_out;       // ||y_m - P||, may be null
     WsHeader *hdr;
     double *partials;            // [grid][2 M]: squared distances to x_A, then of the pulled points to P
+    int grid_a;                  // two-launch schedule: blocks of the distance launch
 };
 
 template <int M>
@@ -44,6 +48,7 @@ struct GeneralColumn {
             ec = __fmaf_rn(a.wn[m], e[m], ec);
         }
         ea = __fmul_rn(ea, 1.0f / (float)M);
+        if (a.uniform) ec = ea;                           // equal weights: the consensus variable IS the average
         const float p = a.push_from_c ? ec : ea;
 #pragma unroll
         for (int m = 0; m < M; ++m) {
@@ -64,6 +69,7 @@ struct GeneralColumn {
             ec = __fmaf_rn(a.wn[m], e[m], ec);
         }
         ea = __fmul_rn(ea, 1.0f / (float)M);
+        if (a.uniform) ec = ea;                           // equal weights: the consensus variable IS the average
         const float p = a.push_from_c ? ec : ea;
         float ub = 0.f;                                   // lambda * mean direction
         if (a.two_term) {
@@ -84,223 +90,247 @@ struct GeneralColumn {
     }
 };
 
+// Four columns of all rows at once (one float4 per row), through the per-column routines.
+template <int M>
+__device__ __forceinline__ void general_distances4(const float4 (&xv)[M], const GeneralArgs &a, float (&pr)[M],
+                                                   float (&pn)[M]) {
+    float xs[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) xs[m] = xv[m].x;
+    GeneralColumn<M>::distances(xs, a, pr, pn);
+#pragma unroll
+    for (int m = 0; m < M; ++m) xs[m] = xv[m].y;
+    GeneralColumn<M>::distances(xs, a, pr, pn);
+#pragma unroll
+    for (int m = 0; m < M; ++m) xs[m] = xv[m].z;
+    GeneralColumn<M>::distances(xs, a, pr, pn);
+#pragma unroll
+    for (int m = 0; m < M; ++m) xs[m] = xv[m].w;
+    GeneralColumn<M>::distances(xs, a, pr, pn);
+}
+template <int M>
+__device__ __forceinline__ void general_update4(float4 (&xv)[M], const GeneralArgs &a, const float *g) {
+    float xs[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) xs[m] = xv[m].x;
+    GeneralColumn<M>::update(xs, a, g);
+#pragma unroll
+    for (int m = 0; m < M; ++m) { xv[m].x = xs[m]; xs[m] = xv[m].y; }
+    GeneralColumn<M>::update(xs, a, g);
+#pragma unroll
+    for (int m = 0; m < M; ++m) { xv[m].y = xs[m]; xs[m] = xv[m].z; }
+    GeneralColumn<M>::update(xs, a, g);
+#pragma unroll
+    for (int m = 0; m < M; ++m) { xv[m].z = xs[m]; xs[m] = xv[m].w; }
+    GeneralColumn<M>::update(xs, a, g);
+#pragma unroll
+    for (int m = 0; m < M; ++m) xv[m].w = xs[m];
+}
+
+// Scalar tail columns (d % 4 of them), one thread.
+template <int M>
+__device__ __forceinline__ void general_tail_distances(const GeneralArgs &a, double (&acc)[2 * M]) {
+    float pr[M], pn[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) pr[m] = pn[m] = 0.f;
+    for (long long i = a.nvec * 4; i < a.d; ++i) {
+        float xs[M];
+#pragma unroll
+        for (int m = 0; m < M; ++m) xs[m] = a.x[m * a.ld + i];
+        GeneralColumn<M>::distances(xs, a, pr, pn);
+    }
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+        acc[m] += (double)pr[m];
+        acc[M + m] += (double)pn[m];
+    }
+}
+template <int M>
+__device__ __forceinline__ void general_tail_update(const GeneralArgs &a, const float *g) {
+    for (long long i = a.nvec * 4; i < a.d; ++i) {
+        float xs[M];
+#pragma unroll
+        for (int m = 0; m < M; ++m) xs[m] = a.x[m * a.ld + i];
+        GeneralColumn<M>::update(xs, a, g);
+#pragma unroll
+        for (int m = 0; m < M; ++m) a.x[m * a.ld + i] = xs[m];
+    }
+}
+
+// Block reduction of the 2M per-thread sums into the block's slot of the partials; `failed`
+// marks the slot negative ("a wait gave up").  Block 0 also stamps the header.
+template <int M, int kWarpsPerBlock>
+__device__ __forceinline__ void general_write_partials(const GeneralArgs &a, const double (&acc)[2 * M], double *s_red,
+                                                       int failed) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+    for (int m = 0; m < 2 * M; ++m) {
+        double sum = warp_sum(acc[m]);
+        if (lane == 0) s_red[warp * 2 * M + m] = sum;
+    }
+    __syncthreads();
+    if (tid < 2 * M) {
+        double sum = 0.0;
+        for (int w = 0; w < kWarpsPerBlock; ++w) sum += s_red[w * 2 * M + tid];
+        a.partials[(long long)blockIdx.x * 2 * M + tid] = failed ? -1.0 : sum;
+    }
+    if (blockIdx.x == 0 && tid == 0) {
+        a.hdr->status = DPPF_OK;
+        a.hdr->magic = kMagic;
+        a.hdr->grid = (int)gridDim.x;
+        a.hdr->M = M;
+    }
+}
+
+// Cross-block sums in block order (identical in every block): fills s_g[m] = lambda / ||y_m - P||
+// (0: no direction), reports both sets of distances, sets *s_flag if any replica differs from the
+// average.  Returns false (in all threads) if nothing is to be written: identical replicas, or a
+// negative mark among the partials (then the status word becomes DPPF_ERR_TIMEOUT).
+template <int M>
+__device__ __forceinline__ bool general_finalise(const GeneralArgs &a, int nblocks, float *s_g, int *s_flag) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    int bad = 0;
+    for (int i = tid; i < nblocks * 2 * M; i += blockDim.x) bad |= (__ldcg(a.partials + i) < 0.0) ? 1 : 0;
+    if (__syncthreads_or(bad)) {
+        if (blockIdx.x == 0 && tid == 0) a.hdr->status = DPPF_ERR_TIMEOUT;
+        return false;
+    }
+    if (tid == 0) *s_flag = 0;
+    __syncthreads();
+    for (int j = warp; j < 2 * M; j += nwarps) {
+        double sum = 0.0;
+        for (int b = lane; b < nblocks; b += 32) sum += __ldcg(a.partials + (long long)b * 2 * M + j);
+        sum = warp_sum(sum);
+        if (lane == 0) {
+            const double nrm = sqrt(sum);
+            if (j < M) {
+                if (nrm > 0.0) *s_flag = 1;               // some replica differs from the average
+                if (blockIdx.x == 0 && a.norms_out) a.norms_out[j] = (float)nrm;
+            } else {
+                s_g[j - M] = (nrm > 0.0) ? (float)((double)a.lambda / nrm) : 0.f;
+                if (blockIdx.x == 0 && a.push_norms_out) a.push_norms_out[j - M] = (float)nrm;
+            }
+        }
+    }
+    __syncthreads();
+    return *s_flag != 0;                                  // identical replicas: nothing moves, x untouched
+}
+
+// One cooperative launch: staged distance pass, grid barrier, staged update pass in reverse.
 template <int M>
 __global__ void __launch_bounds__(kGeneralThreads, 1) general_round_kernel(const GeneralArgs a) {
     constexpr int CH = StagedShape<M>::kChunk;
     constexpr int kStages = StagedShape<M>::kStages;
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    float *ring = reinterpret_cast<float *>(smem_raw);
     __shared__ unsigned long long full[kStages];
     __shared__ double s_red[kGeneralWarps * 2 * M];
     __shared__ float s_g[M];
     __shared__ int s_flag;
     const int tid = threadIdx.x;
-    if (tid == 0) {
-        for (int st = 0; st < kStages; ++st) mbar_init(&full[st], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-
-    const long long d4 = a.nvec * 4;
-    const long long nchunks = (d4 + CH - 1) / CH;
-    const long long n = (nchunks > blockIdx.x) ? (nchunks - 1 - blockIdx.x) / gridDim.x + 1 : 0;
-    unsigned phase = 0;
-    int failed = 0;
-    auto chunk_cols = [&](long long k) -> int {
-        const long long c0 = (blockIdx.x + k * gridDim.x) * CH;
-        return (int)((d4 - c0 < CH) ? (d4 - c0) : CH);
-    };
-    auto issue = [&](long long k) {
-        const int st = (int)(k % kStages);
-        const long long c0 = (blockIdx.x + k * gridDim.x) * CH;
-        const unsigned bytes = (unsigned)chunk_cols(k) * 4u;
-        mbar_expect_tx(&full[st], bytes * M);
-#pragma unroll
-        for (int m = 0; m < M; ++m)
-            bulk_load(ring + ((size_t)st * M + m) * CH, a.x + m * a.ld + c0, bytes, &full[st]);
-    };
+    ChunkRing<M> ring;
+    ring.init(smem_raw, full, a.x, a.ld, a.nvec);
 
     // ---- distance pass: sum (x_m - x_A)^2 and sum (y_m - P)^2 per worker
     double acc[2 * M];
 #pragma unroll
     for (int m = 0; m < 2 * M; ++m) acc[m] = 0.0;
-    if (tid == 0)
-        for (long long k = 0; k < kPrefetchA && k < n; ++k) issue(k);
-    long long k_done = 0;
-    for (long long k = 0; k < n; ++k) {
-        if (tid == 0 && k + kPrefetchA < n) issue(k + kPrefetchA);
-        const int st = (int)(k % kStages);
-        int my_fail = mbar_wait_bounded(&full[st], (phase >> st) & 1u) ? 0 : 1;
-        phase ^= 1u << st;
-        if (!my_fail) {
-            const int cols = chunk_cols(k);
-            const float *sb = ring + (size_t)st * M * CH;
-            float pr[M], pn[M];
-#pragma unroll
-            for (int m = 0; m < M; ++m) pr[m] = pn[m] = 0.f;
-            for (int q = tid * 4; q < cols; q += kGeneralThreads * 4) {
-                float4 xv[M];
-#pragma unroll
-                for (int m = 0; m < M; ++m) xv[m] = *reinterpret_cast<const float4 *>(sb + m * CH + q);
-                float xs[M];
-#pragma unroll
-                for (int m = 0; m < M; ++m) xs[m] = xv[m].x;
-                GeneralColumn<M>::distances(xs, a, pr, pn);
-#pragma unroll
-                for (int m = 0; m < M; ++m) xs[m] = xv[m].y;
-                GeneralColumn<M>::distances(xs, a, pr, pn);
-#pragma unroll
-                for (int m = 0; m < M; ++m) xs[m] = xv[m].z;
-                GeneralColumn<M>::distances(xs, a, pr, pn);
-#pragma unroll
-                for (int m = 0; m < M; ++m) xs[m] = xv[m].w;
-                GeneralColumn<M>::distances(xs, a, pr, pn);
-            }
-#pragma unroll
-            for (int m = 0; m < M; ++m) {
-                acc[m] += (double)pr[m];
-                acc[M + m] += (double)pn[m];
-            }
-        }
-        k_done = k + 1;
-        if (__syncthreads_or(my_fail)) { failed = 1; break; }
-    }
-    if (failed && tid == 0) {
-        const long long hi = (k_done - 1 + kPrefetchA < n - 1) ? k_done - 1 + kPrefetchA : n - 1;
-        for (long long k = k_done; k <= hi; ++k) {
-            const int st = (int)(k % kStages);
-            mbar_wait_bounded(&full[st], (phase >> st) & 1u);
-        }
-    }
-    if (blockIdx.x == 0 && tid == 0) {                    // scalar tail columns
+    int failed = ring_pass<M, StagedShape<M>::kPrefetchA>(ring, a.spin_first, true, 0, [&](float *sb, int k, int) {
+        const int cols = ring.cols(k);
         float pr[M], pn[M];
 #pragma unroll
         for (int m = 0; m < M; ++m) pr[m] = pn[m] = 0.f;
-        for (long long i = d4; i < a.d; ++i) {
-            float xs[M];
+        for (int q = tid * 4; q < cols; q += kGeneralThreads * 4) {
+            float4 xv[M];
 #pragma unroll
-            for (int m = 0; m < M; ++m) xs[m] = a.x[m * a.ld + i];
-            GeneralColumn<M>::distances(xs, a, pr, pn);
+            for (int m = 0; m < M; ++m) xv[m] = *reinterpret_cast<const float4 *>(sb + m * CH + q);
+            general_distances4<M>(xv, a, pr, pn);
         }
 #pragma unroll
         for (int m = 0; m < M; ++m) {
             acc[m] += (double)pr[m];
             acc[M + m] += (double)pn[m];
         }
-    }
-    {
-        const int lane = tid & 31, warp = tid >> 5;
-#pragma unroll
-        for (int m = 0; m < 2 * M; ++m) {
-            double sum = warp_sum(acc[m]);
-            if (lane == 0) s_red[warp * 2 * M + m] = sum;
-        }
-        __syncthreads();
-        if (tid < 2 * M) {
-            double sum = 0.0;
-            for (int w = 0; w < kGeneralWarps; ++w) sum += s_red[w * 2 * M + tid];
-            a.partials[(long long)blockIdx.x * 2 * M + tid] = failed ? -1.0 : sum;
-        }
-        if (blockIdx.x == 0 && tid == 0) {
-            a.hdr->status = DPPF_OK;
-            a.hdr->magic = kMagic;
-            a.hdr->grid = (int)gridDim.x;
-            a.hdr->M = M;
-        }
-    }
+    });
+    if (blockIdx.x == 0 && tid == 0 && !failed) general_tail_distances<M>(a, acc);
+    general_write_partials<M, kGeneralWarps>(a, acc, s_red, failed);
     cg::this_grid().sync();
-
-    {   // did any block give up?
-        int bad = 0;
-        for (int i = tid; i < (int)gridDim.x * 2 * M; i += kGeneralThreads) bad |= (__ldcg(a.partials + i) < 0.0) ? 1 : 0;
-        if (__syncthreads_or(bad)) {
-            if (blockIdx.x == 0 && tid == 0) a.hdr->status = DPPF_ERR_TIMEOUT;
-            return;
-        }
-    }
-    {   // cross-block sums in block order (identical in every block)
-        const int lane = tid & 31, warp = tid >> 5;
-        if (tid == 0) s_flag = 0;
-        __syncthreads();
-        for (int j = warp; j < 2 * M; j += kGeneralWarps) {
-            double sum = 0.0;
-            for (int b = lane; b < (int)gridDim.x; b += 32) sum += __ldcg(a.partials + (long long)b * 2 * M + j);
-            sum = warp_sum(sum);
-            if (lane == 0) {
-                const double nrm = sqrt(sum);
-                if (j < M) {
-                    if (nrm > 0.0) s_flag = 1;            // some replica differs from the average
-                    if (blockIdx.x == 0 && a.norms_out) a.norms_out[j] = (float)nrm;
-                } else {
-                    s_g[j - M] = (nrm > 0.0) ? (float)((double)a.lambda / nrm) : 0.f;
-                    if (blockIdx.x == 0 && a.push_norms_out) a.push_norms_out[j - M] = (float)nrm;
-                }
-            }
-        }
-        __syncthreads();
-        if (!s_flag) return;                              // identical replicas: nothing moves, x untouched
-    }
+    if (!general_finalise<M>(a, (int)gridDim.x, s_g, &s_flag)) return;
 
     // ---- update pass, chunks in reverse, newest chunks reused from the ring
-    const long long resident = (n < kStages) ? n : (long long)kStages;
-    for (long long k = n - 1; k >= 0; --k) {
-        if (tid == 0) {
-            const long long kl = k - kPrefetchB;
-            if (kl >= 0 && kl < n - resident) issue(kl);
+    failed = ring_pass<M, StagedShape<M>::kPrefetchB>(ring, a.spin_later, false, ring.resident(), [&](float *sb, int k, int) {
+        const int cols = ring.cols(k);
+        float *xg = a.x + ring.col0(k);
+        for (int q = tid * 4; q < cols; q += kGeneralThreads * 4) {
+            float4 xv[M];
+#pragma unroll
+            for (int m = 0; m < M; ++m) xv[m] = *reinterpret_cast<const float4 *>(sb + m * CH + q);
+            general_update4<M>(xv, a, s_g);
+#pragma unroll
+            for (int m = 0; m < M; ++m) st_keep(xg + m * a.ld + q, xv[m]);
         }
-        const int st = (int)(k % kStages);
-        int my_fail = 0;
-        if (k < n - resident) {
-            my_fail = mbar_wait_bounded(&full[st], (phase >> st) & 1u) ? 0 : 1;
-            phase ^= 1u << st;
+    });
+    if (failed) {
+        if (tid == 0) a.hdr->status = DPPF_ERR_TIMEOUT;   // x is partly updated
+        return;
+    }
+    if (blockIdx.x == 0 && tid == 0) general_tail_update<M>(a, s_g);
+}
+
+// Two-launch schedule (used when the runtime refuses a cooperative launch, or on request):
+// the same two passes with 128-bit loads straight into registers.
+template <int M>
+__global__ void __launch_bounds__(Tuning<M>::kThreads, Tuning<M>::kBlocksPerSM) general_distance_kernel(const GeneralArgs a) {
+    constexpr int T = Tuning<M>::kThreads;
+    __shared__ double s_red[Tuning<M>::kWarps * 2 * M];
+    float pr[M], pn[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) pr[m] = pn[m] = 0.f;
+    const long long ntiles = (a.nvec + T - 1) / T;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        const long long j = t * T + threadIdx.x;
+        if (j < a.nvec) {
+            float4 xv[M];
+#pragma unroll
+            for (int m = 0; m < M; ++m) xv[m] = ld_keep(a.x + m * a.ld + j * 4);
+            general_distances4<M>(xv, a, pr, pn);
         }
-        if (!my_fail) {
-            const int cols = chunk_cols(k);
-            const long long c0 = (blockIdx.x + k * gridDim.x) * CH;
-            const float *sb = ring + (size_t)st * M * CH;
-            for (int q = tid * 4; q < cols; q += kGeneralThreads * 4) {
+    }
+    double acc[2 * M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+        acc[m] = (double)pr[m];
+        acc[M + m] = (double)pn[m];
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) general_tail_distances<M>(a, acc);
+    general_write_partials<M, Tuning<M>::kWarps>(a, acc, s_red, 0);
+}
+
+template <int M>
+__global__ void __launch_bounds__(Tuning<M>::kThreads, Tuning<M>::kBlocksPerSM) general_update_kernel(const GeneralArgs a) {
+    constexpr int T = Tuning<M>::kThreads;
+    __shared__ float s_g[M];
+    __shared__ int s_flag;
+    if (a.hdr->magic != kMagic || a.hdr->grid != a.grid_a || a.hdr->M != M) {   // not this call's distance launch
+        if (blockIdx.x == 0 && threadIdx.x == 0) a.hdr->status = DPPF_ERR_WORKSPACE;
+        return;
+    }
+    if (!general_finalise<M>(a, a.grid_a, s_g, &s_flag)) return;
+    const long long ntiles = (a.nvec + T - 1) / T;
+    if (ntiles > blockIdx.x) {
+        long long t = blockIdx.x + (ntiles - 1 - blockIdx.x) / gridDim.x * gridDim.x;
+        for (; t >= 0; t -= gridDim.x) {
+            const long long j = t * T + threadIdx.x;
+            if (j < a.nvec) {
                 float4 xv[M];
 #pragma unroll
-                for (int m = 0; m < M; ++m) xv[m] = *reinterpret_cast<const float4 *>(sb + m * CH + q);
-                float xs[M];
+                for (int m = 0; m < M; ++m) xv[m] = ld_last_use(a.x + m * a.ld + j * 4);
+                general_update4<M>(xv, a, s_g);
 #pragma unroll
-                for (int m = 0; m < M; ++m) xs[m] = xv[m].x;
-                GeneralColumn<M>::update(xs, a, s_g);
-#pragma unroll
-                for (int m = 0; m < M; ++m) { xv[m].x = xs[m]; xs[m] = xv[m].y; }
-                GeneralColumn<M>::update(xs, a, s_g);
-#pragma unroll
-                for (int m = 0; m < M; ++m) { xv[m].y = xs[m]; xs[m] = xv[m].z; }
-                GeneralColumn<M>::update(xs, a, s_g);
-#pragma unroll
-                for (int m = 0; m < M; ++m) { xv[m].z = xs[m]; xs[m] = xv[m].w; }
-                GeneralColumn<M>::update(xs, a, s_g);
-#pragma unroll
-                for (int m = 0; m < M; ++m) {
-                    xv[m].w = xs[m];
-                    st_keep(a.x + m * a.ld + c0 + q, xv[m]);
-                }
+                for (int m = 0; m < M; ++m) st_keep(a.x + m * a.ld + j * 4, xv[m]);
             }
         }
-        if (__syncthreads_or(my_fail)) {
-            if (tid == 0) {
-                a.hdr->status = DPPF_ERR_TIMEOUT;
-                const long long kl = k - kPrefetchB;
-                if (k < n - resident && kl >= 0) mbar_wait_bounded(&full[(int)(kl % kStages)], (phase >> (int)(kl % kStages)) & 1u);
-            }
-            return;
-        }
     }
-    if (blockIdx.x == 0 && tid == 0) {
-        for (long long i = d4; i < a.d; ++i) {
-            float xs[M];
-#pragma unroll
-            for (int m = 0; m < M; ++m) xs[m] = a.x[m * a.ld + i];
-            GeneralColumn<M>::update(xs, a, s_g);
-#pragma unroll
-            for (int m = 0; m < M; ++m) a.x[m * a.ld + i] = xs[m];
-        }
-    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) general_tail_update<M>(a, s_g);
 }
 
 }  // namespace

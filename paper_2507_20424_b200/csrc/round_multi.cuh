@@ -1,7 +1,8 @@
 // Several consensus rounds in one persistent launch: the update pass of round k also forms the
 // squared distances round k+1 needs.
 #pragma once
-#include "round_staged.cuh"
+#include "round_register.cuh"
+#include "chunk_ring.cuh"
 
 namespace {
 
@@ -38,44 +39,6 @@ struct RoundsArgs {
     double *partials;             // two buffers of [grid, M], the second at partials + partials_half
     long long partials_half;
     float lambdas[kMaxRoundsPerLaunch];
-};
-
-template <int M>
-struct ChunkRing {
-    static constexpr int CH = StagedShape<M>::kChunk;
-    static constexpr int kStages = StagedShape<M>::kStages;
-    float *ring;                   // [kStages][M][CH]
-    unsigned long long *full;      // one mbarrier per stage
-    const float *x;
-    long long ld, d4, n;           // n = chunks of this block; local chunk k = global chunk blockIdx.x + k gridDim.x
-    unsigned phase;                // bit st: parity of the next wait on stage st
-    long long issued_end;          // thread 0: order index one past the newest copy issued in this pass
-    long long next_wait;           // thread 0: oldest order index whose copy has not been seen to land
-
-    __device__ __forceinline__ long long col0(long long k) const { return (blockIdx.x + k * gridDim.x) * CH; }
-    __device__ __forceinline__ int cols(long long k) const {
-        const long long c0 = col0(k);
-        return (int)((d4 - c0 < CH) ? (d4 - c0) : CH);
-    }
-    __device__ __forceinline__ float *stage(long long k) const { return ring + (size_t)(k % kStages) * M * CH; }
-    // lanes 0..M-1 of warp 0 (or lane 0 alone when M > 32 cannot happen: M <= 16): one row copy each
-    __device__ __forceinline__ void issue(long long k) {
-        const int st = (int)(k % kStages);
-        const unsigned bytes = (unsigned)cols(k) * 4u;
-        const int lane = threadIdx.x;
-        if (lane == 0) mbar_expect_tx(&full[st], bytes * M);
-        __syncwarp();
-        if (lane < M) bulk_load(ring + ((size_t)st * M + lane) * CH, x + lane * ld + col0(k), bytes, &full[st]);
-    }
-    __device__ __forceinline__ bool wait(long long k, int limit) {
-        const int st = (int)(k % kStages);
-        for (int spins = 0; spins < limit; ++spins)
-            if (mbar_try_wait(&full[st], (phase >> st) & 1u)) {
-                phase ^= 1u << st;
-                return true;
-            }
-        return false;
-    }
 };
 
 // One chunk in shared memory: optional update with coefficients c (written to x and, if asked,
@@ -124,25 +87,9 @@ __global__ void __launch_bounds__(kStagedThreads, 1) rounds_kernel_staged(const 
     __shared__ double s_red[kStagedWarps * M];
     __shared__ float s_c[M];
     const int tid = threadIdx.x;
-    if (tid == 0) {
-        for (int st = 0; st < kStages; ++st) mbar_init(&full[st], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-
     ChunkRing<M> ring;
-    ring.ring = reinterpret_cast<float *>(smem_raw);
-    ring.full = full;
-    ring.x = a.x;
-    ring.ld = a.ld;
-    ring.d4 = a.nvec * 4;
-    {
-        const long long nchunks = (ring.d4 + ChunkRing<M>::CH - 1) / ChunkRing<M>::CH;
-        ring.n = (nchunks > blockIdx.x) ? (nchunks - 1 - blockIdx.x) / gridDim.x + 1 : 0;
-    }
-    ring.phase = 0;
-    const long long n = ring.n;
-    const long long resident_max = (n < kStages) ? n : (long long)kStages;
+    ring.init(smem_raw, full, a.x, a.ld, a.nvec);
+    const int n = ring.n;
 
     // tail columns (d % 4 of them) go through the scalar routines, which take the single-round arguments
     RoundArgs tail_args;
@@ -153,44 +100,25 @@ __global__ void __launch_bounds__(kStagedThreads, 1) rounds_kernel_staged(const 
     const int R = a.n_rounds;
     for (int p = 0; p <= R; ++p) {
         const bool first = (p == 0), last = (p == R), fwd = !(p & 1);
-        const int prefetch = first ? kPrefetchA : kPrefetchB;
-        const int limit = first ? a.spin_first : a.spin_later;
-        const long long resident = first ? 0 : resident_max;   // leading chunks of this pass still in the ring
         double acc[M];
 #pragma unroll
         for (int m = 0; m < M; ++m) acc[m] = 0.0;
-        int failed = 0;
-
-        ring.issued_end = ring.next_wait = resident;
-        if (tid < 32)
-            for (long long j = resident; j < prefetch && j < n; ++j) {
-                ring.issue(fwd ? j : n - 1 - j);
-                ring.issued_end = j + 1;
-            }
-        for (long long i = 0; i < n; ++i) {
-            const long long k = fwd ? i : n - 1 - i;
-            const long long j = i + prefetch;                    // order index to fetch now
-            if (tid < 32 && j >= resident && j < n) {            // its stage held order index j - kStages: consumed
-                ring.issue(fwd ? j : n - 1 - j);
-                ring.issued_end = j + 1;
-            }
-            int my_fail = 0;
-            if (i >= resident) {
-                my_fail = ring.wait(k, limit) ? 0 : 1;
-                if (!my_fail) ring.next_wait = i + 1;
-            }
-            if (!my_fail) {
+        int failed;
+        if (first) {
+            failed = ring_pass<M, StagedShape<M>::kPrefetchA>(ring, a.spin_first, fwd, 0, [&](float *sb, int k, int) {
+                chunk_body<M, false>(sb, nullptr, 0, ring.cols(k), s_c, false, true, acc);
+            });
+        } else if (last) {
+            failed = ring_pass<M, StagedShape<M>::kPrefetchB>(ring, a.spin_later, fwd, ring.resident(), [&](float *sb, int k, int) {
+                chunk_body<M, true>(sb, a.x + ring.col0(k), a.ld, ring.cols(k), s_c, false, false, acc);
+            });
+        } else {
+            failed = ring_pass<M, StagedShape<M>::kPrefetchB>(ring, a.spin_later, fwd, ring.resident(), [&](float *sb, int k, int i) {
                 // chunks this pass handles last are the first of the next pass: keep them current in the ring
-                const bool write_back = !last && i >= n - kStages;
-                if (first) chunk_body<M, false>(ring.stage(k), nullptr, 0, ring.cols(k), s_c, false, true, acc);
-                else chunk_body<M, true>(ring.stage(k), a.x + ring.col0(k), a.ld, ring.cols(k), s_c, write_back, !last, acc);
+                const bool write_back = i >= n - kStages;
+                chunk_body<M, true>(sb, a.x + ring.col0(k), a.ld, ring.cols(k), s_c, write_back, true, acc);
                 if (write_back) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            }
-            if (__syncthreads_or(my_fail)) { failed = 1; break; }  // block-uniform decision
-        }
-        if (failed && tid == 0) {
-            // copies still in flight get the full poll budget to land before the block moves on
-            for (long long j = ring.next_wait; j < ring.issued_end; ++j) ring.wait(fwd ? j : n - 1 - j, kSpinLimit);
+            });
         }
         if (blockIdx.x == 0 && tid == 0 && !failed) {
             if (!first) tail_update<M>(tail_args, s_c);
@@ -260,13 +188,9 @@ __global__ void __launch_bounds__(kStagedThreads, 1) rounds_kernel_staged(const 
     }
 }
 
-}  // namespace
-
-namespace {
-
-// ---------------------------------------------------------------- n rounds, register-resident (9 <= M <= 16)
-// Same schedule of passes with 128-bit loads straight into registers (the shared-memory ring
-// pays off only up to eight rows).  Per-thread fp32 sums per pass, fp64 from the warp upwards.
+// ---------------------------------------------------------------- n rounds, register-resident
+// Same schedule of passes with 128-bit loads straight into registers, for when the ring cannot
+// be used.  Per-thread fp32 sums per pass, fp64 from the warp upwards.
 template <int M, int U, bool kUpdate>
 __device__ __forceinline__ void register_pass(const RoundsArgs &a, const float *c, bool fwd, bool accumulate,
                                               float (&acc)[M]) {

@@ -14,7 +14,7 @@ namespace {
 template <int M>
 struct Tuning {
     static constexpr int kThreads =
-        (M <= 2) ? 320 : (M == 3) ? 384 : (M == 4) ? 320 : (M == 5) ? 288 : (M == 6) ? 224 :
+        (M <= 2) ? 320 : (M == 3) ? 384 : (M == 4) ? 320 : (M == 5) ? 256 : (M == 6) ? 224 :
         (M <= 8) ? 192 : (M == 9) ? 320 : (M == 10) ? 288 : (M <= 12) ? 256 : 224;
     static constexpr int kBlocksPerSM = (M <= 8) ? 2 : 1;
     static constexpr int kUnrollA = (M <= 2) ? 4 : (M <= 8) ? 2 : 1;      // distance pass
@@ -160,11 +160,12 @@ __device__ __forceinline__ void distance_pass(const RoundArgs &a, double *s_red 
 }
 
 // Cross-block sum in block order, identical in every block; fills s_c[M] and reports r_m.
-// Returns false if the workspace header does not describe this launch.
+// Returns false if the workspace header does not describe this launch.  With a.hdr == nullptr
+// the partials are the caller's own M sums (nblocks == 1) and there is no header to check.
 __device__ __forceinline__ bool finalise(const RoundArgs &a, int M, int nblocks, float *s_c, int *s_ok) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0)
-        *s_ok = (a.hdr->magic == kMagic && a.hdr->grid == nblocks && a.hdr->M == M) ? 1 : 0;
+        *s_ok = (!a.hdr || (a.hdr->magic == kMagic && a.hdr->grid == nblocks && a.hdr->M == M)) ? 1 : 0;
     const int nwarps = blockDim.x >> 5;
     for (int m = warp; m < M; m += nwarps) {
         double s = 0.0;
@@ -174,7 +175,7 @@ __device__ __forceinline__ bool finalise(const RoundArgs &a, int M, int nblocks,
             float r;
             s_c[m] = coefficient(s, a.alpha, a.lambda, &r);
             if (blockIdx.x == 0) {
-                a.norms_stage[m] = r;
+                if (a.norms_stage) a.norms_stage[m] = r;
                 if (a.norms_out) a.norms_out[m] = r;
             }
         }
@@ -184,9 +185,8 @@ __device__ __forceinline__ bool finalise(const RoundArgs &a, int M, int nblocks,
     return *s_ok != 0;
 }
 
-template <int M, int U>
+template <int M, int U, int T = Tuning<M>::kThreads>
 __device__ __forceinline__ void update_pass(const RoundArgs &a, const float *s_c) {
-    constexpr int T = Tuning<M>::kThreads;
     const long long tile_vecs = (long long)T * U;
     const long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
     const float *c = s_c;
@@ -236,6 +236,18 @@ update_kernel(const RoundArgs a, int nblocks_a) {
     __shared__ int s_ok;
     if (!finalise(a, M, nblocks_a, s_c, &s_ok)) return;
     update_pass<M, (kAfterLocalStep ? Tuning<M>::kUnrollBFused : Tuning<M>::kUnrollB)>(a, s_c);
+}
+
+// Per-worker totals of the per-block partial sums, in block order (the order finalise uses):
+// what a column shard contributes to the squared distances.  One block of up to 16 warps.
+__global__ void sum_partials_kernel(const double *partials, int nblocks, int M, double *sums_out) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    for (int m = warp; m < M; m += nwarps) {
+        double s = 0.0;
+        for (int b = lane; b < nblocks; b += 32) s += __ldcg(partials + (long long)b * M + m);
+        s = warp_sum(s);
+        if (lane == 0) sums_out[m] = s;
+    }
 }
 
 // One persistent launch: distance pass, grid-wide barrier, update pass.  Launched with

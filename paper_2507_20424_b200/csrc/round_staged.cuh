@@ -1,10 +1,11 @@
 // Staged persistent round kernel: rows streamed through a shared-memory ring by bulk async copies.
 #pragma once
 #include "round_register.cuh"
+#include "chunk_ring.cuh"
 
 namespace {
 
-// ---------------------------------------------------------------- staged persistent kernel (default, M <= 16)
+// ---------------------------------------------------------------- staged persistent kernel, one round (default for M <= 8)
 // One block per SM keeps a ring of up to kMaxStages shared-memory stages; a stage holds the same
 // column chunk of all M rows (about 32 KB).  One thread fills stages with 1-D bulk async
 // copies (cp.async.bulk, completion on an mbarrier); all threads then read the chunk from
@@ -19,54 +20,11 @@ namespace {
 // with a negative value, every block then sees the mark after the grid barrier, nobody
 // writes x, and the status word reports DPPF_ERR_TIMEOUT.
 
-constexpr int kStagedThreads = 256;
-constexpr int kStagedWarps = kStagedThreads / 32;
-constexpr int kMaxStages = 6;
-constexpr int kPrefetchA = 3;
-constexpr int kPrefetchB = 1;
-constexpr int kSpinLimit = 1 << 22;   // mbarrier try_wait polls before a wait gives up (~ a second)
-
-template <int M>
-struct StagedShape {
-    // columns per stage and row: a stage of about 32 KB (40 KB measured best for M = 8)
-    static constexpr int kChunk = (M == 8) ? 1280 : ((8192 / M) / 128) * 128;
-    static constexpr size_t kStageFloats = (size_t)M * kChunk;
-    static constexpr int kFit = (int)((200 * 1024) / (kStageFloats * sizeof(float)));
-    static constexpr int kStages = kFit < kMaxStages ? kFit : kMaxStages;
-    static constexpr size_t kSmemBytes = (size_t)kStages * kStageFloats * sizeof(float);
-    static_assert(kStages > kPrefetchA, "ring must be deeper than the prefetch distance");
-};
-
-__device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(unsigned long long *bar, int count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned long long *bar, unsigned parity) {
-    unsigned ok;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: false if the phase did not complete within kSpinLimit polls.
-__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long *bar, unsigned parity) {
-    for (int spins = 0; spins < kSpinLimit; ++spins)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-// global -> shared bulk copy; dst, src 16-byte aligned, bytes a multiple of 16.
-__device__ __forceinline__ void bulk_load(void *dst_smem, const void *src, unsigned bytes, unsigned long long *bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_addr(dst_smem)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
-}
-
 template <int M>
 __global__ void __launch_bounds__(kStagedThreads, 1) round_kernel_staged(const RoundArgs a) {
     constexpr int CH = StagedShape<M>::kChunk;
     constexpr int kStages = StagedShape<M>::kStages;
+    constexpr int kPrefetchA = StagedShape<M>::kPrefetchA, kPrefetchB = StagedShape<M>::kPrefetchB;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     float *ring = reinterpret_cast<float *>(smem_raw);             // [kStages][M][CH]
     __shared__ unsigned long long full[kStages];
@@ -107,13 +65,16 @@ __global__ void __launch_bounds__(kStagedThreads, 1) round_kernel_staged(const R
     for (int m = 0; m < M; ++m) acc[m] = 0.0;
     if (tid == 0)
         for (long long k = 0; k < kPrefetchA && k < n; ++k) issue(k);
-    long long k_done = 0;                                           // chunks consumed so far
+    long long k_done = 0;                                           // chunks this thread saw land
+    long long k_fail = 0;                                           // iteration in which the block gave up
     for (long long k = 0; k < n; ++k) {
+        k_fail = k;
         if (tid == 0 && k + kPrefetchA < n) issue(k + kPrefetchA);
         const int st = (int)(k % kStages);
-        int my_fail = mbar_wait_bounded(&full[st], (phase >> st) & 1u) ? 0 : 1;
-        phase ^= 1u << st;
+        int my_fail = mbar_wait_bounded(&full[st], (phase >> st) & 1u, a.spin_first) ? 0 : 1;
         if (!my_fail) {
+            phase ^= 1u << st;
+            k_done = k + 1;
             const int cols = chunk_cols(k);
             const float *sb = ring + (size_t)st * M * CH;
             float part[M];
@@ -130,15 +91,15 @@ __global__ void __launch_bounds__(kStagedThreads, 1) round_kernel_staged(const R
 #pragma unroll
             for (int m = 0; m < M; ++m) acc[m] += (double)part[m];
         }
-        k_done = k + 1;
         if (__syncthreads_or(my_fail)) { failed = 1; break; }      // block-uniform decision
     }
     if (failed && tid == 0) {
-        // give this block's copies still in flight a bounded chance to land before moving on
-        const long long hi = (k_done - 1 + kPrefetchA < n - 1) ? k_done - 1 + kPrefetchA : n - 1;
+        // copies still in flight (from the first chunk this thread did not see land) get the full
+        // poll budget before the block moves on
+        const long long hi = (k_fail + kPrefetchA < n - 1) ? k_fail + kPrefetchA : n - 1;
         for (long long k = k_done; k <= hi; ++k) {
             const int st = (int)(k % kStages);
-            mbar_wait_bounded(&full[st], (phase >> st) & 1u);
+            mbar_wait_bounded(&full[st], (phase >> st) & 1u, kSpinLimit);
         }
     }
     if (blockIdx.x == 0 && tid == 0) {
@@ -192,8 +153,8 @@ __global__ void __launch_bounds__(kStagedThreads, 1) round_kernel_staged(const R
         const int st = (int)(k % kStages);
         int my_fail = 0;
         if (k < n - resident) {
-            my_fail = mbar_wait_bounded(&full[st], (phase >> st) & 1u) ? 0 : 1;
-            phase ^= 1u << st;
+            my_fail = mbar_wait_bounded(&full[st], (phase >> st) & 1u, a.spin_later) ? 0 : 1;
+            if (!my_fail) phase ^= 1u << st;
         }
         if (!my_fail) {
             const int cols = chunk_cols(k);
@@ -213,8 +174,11 @@ __global__ void __launch_bounds__(kStagedThreads, 1) round_kernel_staged(const R
         if (__syncthreads_or(my_fail)) {
             if (tid == 0) {
                 a.hdr->status = DPPF_ERR_TIMEOUT;                   // x is partly updated
-                const long long kl = k - kPrefetchB;                // the one copy that may still be in flight
-                if (k < n - resident && kl >= 0) mbar_wait_bounded(&full[(int)(kl % kStages)], (phase >> (int)(kl % kStages)) & 1u);
+                // the copies that may still be in flight: chunk k (unless this thread saw it land) and k - 1
+                if (my_fail) mbar_wait_bounded(&full[st], (phase >> st) & 1u, kSpinLimit);
+                const long long kl = k - kPrefetchB;
+                if (kl >= 0 && kl < n - resident)
+                    mbar_wait_bounded(&full[(int)(kl % kStages)], (phase >> (int)(kl % kStages)) & 1u, kSpinLimit);
             }
             return;
         }
