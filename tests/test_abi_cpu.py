@@ -102,6 +102,18 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert rounds(X, 4, 64, 64, float("nan"), 0.01, None, 2, None, WS, big, None) == b.ERR_INVALID_ARG
     assert rounds(X, 4, 64, 64, 0.1, 0.01, None, 2, None, WS, 16, None) == b.ERR_WORKSPACE
     assert rounds(X, 4, 64, 64, 0.1, 0.01, None, 2, X + 64, WS, big, None) == b.ERR_INVALID_ARG   # norms inside x
+    SUMS = 0x50000000
+    dp, uf = lib.dppf_distance_partials, lib.dppf_update_from_sums
+    assert dp(None, 4, 64, 64, SUMS, WS, big, None) == b.ERR_INVALID_ARG
+    assert dp(X, 4, 64, 64, None, WS, big, None) == b.ERR_INVALID_ARG
+    assert dp(X, 4, 64, 64, SUMS + 4, WS, big, None) == b.ERR_INVALID_ARG             # fp64 alignment
+    assert dp(X, 4, 64, 64, SUMS, WS, 16, None) == b.ERR_WORKSPACE
+    assert dp(X, 4, 64, 64, X + 8, WS, big, None) == b.ERR_INVALID_ARG                # sums inside x
+    assert uf(X, 4, 64, 64, 0.1, 0.01, None, None, None) == b.ERR_INVALID_ARG
+    assert uf(X, 4, 64, 64, float("inf"), 0.01, SUMS, None, None) == b.ERR_INVALID_ARG
+    assert uf(X, 4, 60, 60, 0.1, 0.01, SUMS, None, None) == b.ERR_ALIGNMENT
+    assert lib.dppf_consensus_general_ex(X, 4, 64, 64, 0.1, 0.01, None, 0, 0, None, None, WS, big, 2, None) == b.ERR_INVALID_ARG
+    assert lib.dppf_consensus_static(X, 4, 64, 64, float("nan"), 0.01, None, None) == b.ERR_INVALID_ARG
     assert lib.dppf_consensus_rounds_ex(X, 4, 64, 64, 0.1, 0.01, None, 2, None, WS, big, 9, None) == b.ERR_INVALID_ARG
 
 

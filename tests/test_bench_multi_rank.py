@@ -70,3 +70,56 @@ def test_reference_arm_prints_one_line_and_other_ranks_stay_silent():
     assert out["impl"] == "reference" and out["unit"] == "rounds/s" and out["value"] > 0
     assert out["cpu_baseline"]["kind"] == "oracle" and out["cpu_baseline"]["cores"] >= 1
     assert out["e2e"]["h2d_bytes_per_step"] == 0 and out["e2e"]["d2h_bytes_per_step"] == 0
+
+
+SHARD_WORKER = r"""
+import os, sys, json
+sys.path.insert(0, sys.argv[1])
+import numpy as np
+import torch, torch.distributed as dist
+import bench, oracle
+from paper_2507_20424_b200 import inputs
+rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+dist.init_process_group("gloo")
+# column shards of ONE replica set (same seed on every rank)
+w = inputs.WORKLOADS["C1"].scaled(10_007)
+x = inputs.replicas(w)
+lo, hi = bench.column_shard(w.d, world, rank)
+# this rank's share of the sums of squares: the oracle's distances on its own columns, squared
+_, r_shard = oracle.consensus(np.ascontiguousarray(x[:, lo:hi]), w.alpha, 0.0)
+sums = torch.from_numpy(r_shard ** 2)
+dist.all_reduce(sums)                                   # the one exchange of a column-sharded round
+spans = [None] * world
+dist.all_gather_object(spans, (lo, hi))
+_, r_full = oracle.consensus(x, w.alpha, 0.0, d=w.d)
+if rank == 0:
+    print(json.dumps({"spans": spans, "d": w.d, "r": np.sqrt(sums.numpy()).tolist(), "r_full": r_full.tolist()}))
+dist.destroy_process_group()
+"""
+
+
+def test_two_ranks_column_shards_and_sum_exchange(tmp_path):
+    """Column shards tile [0, d) on 128-byte boundaries, and adding the shards' sums of squares
+    over the ranks gives the distances of the whole vector."""
+    script = tmp_path / "shard_worker.py"
+    script.write_text(SHARD_WORKER)
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+           "--master-addr", "127.0.0.1", "--master-port", "29534", str(script), ROOT]
+    run = subprocess.run(cmd, capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert run.returncode == 0, run.stderr[-2000:]
+    out = json.loads([l for l in run.stdout.splitlines() if l.startswith("{")][-1])
+    (lo0, hi0), (lo1, hi1) = out["spans"]
+    assert lo0 == 0 and hi0 == lo1 and hi1 == out["d"] and lo1 % 32 == 0
+    assert out["r"] == pytest.approx(out["r_full"], rel=1e-12)
+
+
+def test_column_shard_covers_every_column_once():
+    sys.path.insert(0, ROOT)
+    import bench
+    for d in (1, 31, 32, 33, 1000, 86_567_656):
+        for world in (1, 2, 3, 8):
+            spans = [bench.column_shard(d, world, r) for r in range(world)]
+            assert spans[0][0] == 0 and spans[-1][1] == d
+            for (lo, hi), (lo2, _) in zip(spans[:-1], spans[1:]):
+                assert hi == lo2 and lo <= hi
+            assert all(lo % 32 == 0 or lo == hi for lo, hi in spans)      # non-empty shards start on 128 bytes

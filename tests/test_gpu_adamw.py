@@ -22,8 +22,10 @@ def close(got, ref):
     return np.all(np.abs(got.astype(np.float64) - ref) <= 2e-6 * np.abs(ref).max() + 1e-5 * np.abs(ref))
 
 
-@pytest.mark.parametrize("M,d,tau", [(1, 1003, 2), (2, 33, 3), (4, 1_000_003, 4), (8, 200_001, 2), (16, 50_001, 2), (5, 7, 1)])
-def test_adamw_steps_then_fused_round(oracle, M, d, tau):
+@pytest.mark.parametrize("path", [2, 1])          # one cooperative launch / two launches
+@pytest.mark.parametrize("M,d,tau", [(1, 1003, 2), (2, 33, 3), (4, 1_000_003, 4), (8, 200_001, 2), (16, 50_001, 2), (5, 7, 1),
+                                     (7, 300_001, 2), (12, 150_003, 2)])
+def test_adamw_steps_then_fused_round(oracle, M, d, tau, path):
     import torch
     _, binding = require_gpu()
     w = workload(M, d)
@@ -39,7 +41,7 @@ def test_adamw_steps_then_fused_round(oracle, M, d, tau):
         binding.dppf_adamw_step(x, a, b, to_dev(grads[t]), step=t + 1, d=d, **HP)
     g_last = to_dev(grads[-1])
     binding.dppf_adamw_step_and_consensus(x, a, b, g_last, step=tau, alpha=w.alpha, lam=w.lam,
-                                          norms_out=norms, ws=ws, d=d, **HP)
+                                          norms_out=norms, ws=ws, d=d, path=path, **HP)
     assert binding.dppf_device_status(ws) == binding.OK
     got_x, got_a, got_b = x.cpu().numpy(), a.cpu().numpy(), b.cpu().numpy()
     assert_parity(got_x, norms.cpu().numpy(), ref, r_ref, d)
@@ -68,6 +70,23 @@ def test_fused_matches_step_then_round():
     assert same_bits(ba.cpu().numpy()[:, :w.d], bb.cpu().numpy()[:, :w.d])
     np.testing.assert_allclose(nb.cpu().numpy(), na.cpu().numpy(), rtol=2e-6)
     assert np.max(np.abs(xa.cpu().numpy()[:, :w.d].astype(np.float64) - xb.cpu().numpy()[:, :w.d])) <= 1e-7
+
+
+@pytest.mark.parametrize("M", [4, 8, 16])
+def test_both_schedules_agree_bit_for_bit(M):
+    import torch
+    _, binding = require_gpu()
+    w = workload(M, 1_200_003)
+    x_np, z, g = inputs.replicas(w), inputs.zeros_like_rows(w), inputs.gradients(w, 0)
+    x_np[:, :w.d] += inputs.gradients(w, 7)[:, :w.d]
+    outs = []
+    for path in (2, 1):
+        x, a, b = to_dev(x_np), to_dev(z), to_dev(z)
+        n = torch.zeros(M, device="cuda")
+        binding.dppf_adamw_step_and_consensus(x, a, b, to_dev(g), step=3, alpha=w.alpha, lam=w.lam, norms_out=n,
+                                              d=w.d, path=path, **HP)
+        outs.append((x.cpu().numpy()[:, :w.d], a.cpu().numpy()[:, :w.d], b.cpu().numpy()[:, :w.d], n.cpu().numpy()))
+    assert all(same_bits(p, q) for p, q in zip(*outs))
 
 
 def test_adamw_rejects_bad_arguments():

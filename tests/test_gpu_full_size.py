@@ -141,3 +141,133 @@ def test_rows_longer_than_2_to_31_columns(oracle, path):
     assert torch.isnan(x[:, d:]).all()
     del x, blk
     torch.cuda.empty_cache()
+
+
+# ---------------------------------------------------------------- several rounds per launch
+
+def test_c4_hundred_rounds_in_one_call(oracle):
+    """The 100 back-to-back rounds of the ViT-B/16-sized workload as ONE dppf_consensus_rounds call
+    (what the benchmark's multi_round figure times): the replicas after round 100 and the
+    distances before every one of the 100 rounds against the oracle iterated 100 times."""
+    import torch
+    _, binding = require_gpu()
+    w = inputs.WORKLOADS["C4"]
+    x_np = inputs.replicas(w)
+    ref, rs = x_np, []
+    for _ in range(w.rounds):
+        ref, r_ref, _ = oracle.consensus_blocked(ref, w.alpha, w.lam, d=w.d)
+        rs.append(r_ref)
+    rs = np.array(rs)
+    outs = []
+    for _ in range(2):
+        x = to_dev(x_np)
+        norms = torch.full((w.rounds, w.M), -1.0, device="cuda")
+        ws = binding.alloc_workspace(w.M, w.d)
+        binding.dppf_consensus_rounds(x, w.alpha, w.lam, w.rounds, norms_out=norms, ws=ws, d=w.d)
+        assert binding.dppf_device_status(ws) == binding.OK
+        outs.append((x.cpu().numpy(), norms.cpu().numpy()))
+        del x
+        torch.cuda.empty_cache()
+    got, norms = outs[0]
+    assert_parity(got, norms[-1], ref, rs[-1], w.d)
+    assert np.all(np.abs(norms - rs) <= 1e-5 * rs)
+    assert_pad_untouched(got, w.d)
+    assert same_bits(got[:, :w.d], outs[1][0][:, :w.d]) and same_bits(norms, outs[1][1])      # run to run
+    np.testing.assert_allclose(norms[0], w.drift_std * np.sqrt(w.d * (w.M - 1) / w.M), rtol=0.01)
+
+
+@pytest.mark.parametrize("name,n", [("C1", 100), ("C2", 5), ("C5", 3)])
+def test_rounds_in_one_call_other_workloads(oracle, name, n):
+    import torch
+    _, binding = require_gpu()
+    w = inputs.WORKLOADS[name]
+    x_np = inputs.replicas(w)
+    ref, rs = x_np, []
+    for _ in range(n):
+        ref, r_ref, _ = oracle.consensus_blocked(ref, w.alpha, w.lam, d=w.d)
+        rs.append(r_ref)
+    rs = np.array(rs)
+    x = to_dev(x_np)
+    norms = torch.full((n, w.M), -1.0, device="cuda")
+    ws = binding.alloc_workspace(w.M, w.d)
+    binding.dppf_consensus_rounds(x, w.alpha, w.lam, n, norms_out=norms, ws=ws, d=w.d)
+    assert binding.dppf_device_status(ws) == binding.OK
+    got, norms = x.cpu().numpy(), norms.cpu().numpy()
+    del x
+    torch.cuda.empty_cache()
+    assert_parity(got, norms[-1], ref, rs[-1], w.d)
+    assert np.all(np.abs(norms - rs) <= 1e-5 * rs)
+    assert_pad_untouched(got, w.d)
+
+
+# ---------------------------------------------------------------- general round and AdamW at full size
+
+@pytest.mark.parametrize("name,wkind,push_from,two_term", [("C4", "random", "consensus", True),
+                                                           ("C2", "leader", "consensus", False),
+                                                           ("C5", "random", "average", True)])
+def test_general_round_full_size(oracle, name, wkind, push_from, two_term):
+    """Weighted consensus variable / a leader, push from x_A or x_C, one or both gradient terms,
+    at the workloads' full sizes (every block wraps its ring many times)."""
+    import torch
+    _, binding = require_gpu()
+    w = inputs.WORKLOADS[name]
+    x_np = inputs.replicas(w)
+    if wkind == "leader":
+        wts = np.zeros(w.M)
+        wts[w.M // 2] = 1.0
+    else:
+        wts = np.random.default_rng(7).random(w.M) + 0.05
+    ref, r_ref, n_ref = oracle.consensus_general(x_np, w.alpha, w.lam, wts, push_from, two_term, d=w.d)
+    x = to_dev(x_np)
+    r = torch.full((w.M,), -1.0, device="cuda")
+    n = torch.full((w.M,), -1.0, device="cuda")
+    ws = binding.alloc_workspace(w.M, w.d)
+    binding.dppf_consensus_general(x, w.alpha, w.lam, wts, {"average": 0, "consensus": 1}[push_from], two_term,
+                                   norms_out=r, push_norms_out=n, ws=ws, d=w.d)
+    assert binding.dppf_device_status(ws) == binding.OK
+    got = x.cpu().numpy()
+    del x
+    torch.cuda.empty_cache()
+    assert_parity(got, r.cpu().numpy(), ref, r_ref, w.d)
+    assert np.all(np.abs(n.cpu().numpy() - n_ref) <= 1e-5 * n_ref)
+    assert_pad_untouched(got, w.d)
+
+
+def test_adamw_steps_then_fused_round_at_vit_size(oracle):
+    """The paper's ViT setting (AdamW, lr 5e-4, weight decay 0.01) at the ViT-B/16-sized
+    workload: one stand-alone AdamW step, then the second step fused with the round; replicas,
+    both moment buffers and the distances against the fp64 oracle."""
+    import torch
+    from dataclasses import replace
+    _, binding = require_gpu()
+    hp = dict(lr=5e-4, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    w = replace(inputs.WORKLOADS["C4"], grad_std=1e-2, alpha=0.9, lam=0.09)
+    x_np = inputs.replicas(w)
+    x = to_dev(x_np)
+    a, b = binding.alloc_rows(w.M, w.d, fill=0.0), binding.alloc_rows(w.M, w.d, fill=0.0)
+    x64 = np.array(x_np[:, :w.d], dtype=np.float64)
+    a64, b64 = np.zeros_like(x64), np.zeros_like(x64)
+    norms = torch.zeros(w.M, device="cuda")
+    ws = binding.alloc_workspace(w.M, w.d)
+    for t in range(2):
+        g_np = inputs.gradients(w, t)
+        x64, a64, b64 = oracle.adamw_steps_f64(x64, a64, b64, [g_np[:, :w.d]], first_step=t + 1, **hp)
+        g = to_dev(g_np)
+        if t == 0:
+            binding.dppf_adamw_step(x, a, b, g, step=1, d=w.d, **hp)
+        else:
+            binding.dppf_adamw_step_and_consensus(x, a, b, g, step=2, alpha=w.alpha, lam=w.lam, norms_out=norms,
+                                                  ws=ws, d=w.d, **hp)
+        torch.cuda.synchronize()
+        del g, g_np
+    ref, r_ref = oracle.consensus_f64(x64, w.alpha, w.lam)
+    del x64
+    assert binding.dppf_device_status(ws) == binding.OK
+    got_x = x.cpu().numpy()
+    assert_parity(got_x, norms.cpu().numpy(), ref, r_ref, w.d)
+    assert_pad_untouched(got_x, w.d)
+    for got, want in ((a.cpu().numpy()[:, :w.d], a64), (b.cpu().numpy()[:, :w.d], b64)):
+        err = np.abs(got.astype(np.float64) - want)
+        assert np.all(err <= 2e-6 * np.abs(want).max() + 1e-5 * np.abs(want))
+    del x, a, b
+    torch.cuda.empty_cache()

@@ -15,7 +15,10 @@ def replicas(M, d, seed, base=0.02, drift=1e-3):
     return padded((x0[None, :] + rng.standard_normal((M, d)) * drift).astype(np.float32))
 
 
-def run(binding, x_np, d, alpha, lam, weights, push_from, two_term):
+PATHS = {"staged": 3, "two_kernel": 1}
+
+
+def run(binding, x_np, d, alpha, lam, weights, push_from, two_term, path=0):
     import torch
     M = x_np.shape[0]
     x = to_dev(x_np)
@@ -24,7 +27,7 @@ def run(binding, x_np, d, alpha, lam, weights, push_from, two_term):
     ws = binding.alloc_workspace(M, d)
     binding.dppf_consensus_general(x, alpha, lam, weights,
                                    {"average": 0, "consensus": 1}[push_from], two_term,
-                                   norms_out=r, push_norms_out=n, ws=ws, d=d)
+                                   norms_out=r, push_norms_out=n, ws=ws, d=d, path=path)
     assert binding.dppf_device_status(ws) == binding.OK
     return x.cpu().numpy(), r.cpu().numpy(), n.cpu().numpy()
 
@@ -39,21 +42,58 @@ def weights_for(kind, M, seed):
     return np.random.default_rng(seed).random(M) + 0.05
 
 
+def check(got, r, n, ref, r_ref, n_ref, d):
+    assert_parity(got, r, ref, r_ref, d)
+    assert np.all(np.abs(n - n_ref) <= 1e-5 * n_ref + 1e-30)
+    assert np.all(n[n_ref == 0.0] == 0.0)
+    assert_pad_untouched(got, d)
+
+
+@pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("two_term", [False, True])
 @pytest.mark.parametrize("push_from", ["average", "consensus"])
 @pytest.mark.parametrize("wkind", ["none", "random", "leader"])
 @pytest.mark.parametrize("M,d", [(1, 1000), (2, 5), (3, 4099), (4, 300_001), (5, 70_003), (8, 1_000_003),
                                  (16, 200_001)])
-def test_general_round_matches_oracle(oracle, M, d, wkind, push_from, two_term):
+def test_general_round_matches_oracle(oracle, M, d, wkind, push_from, two_term, path):
     _, binding = require_gpu()
     x = replicas(M, d, seed=M * 31 + d % 97)
     w = weights_for(wkind, M, d)
     ref, r_ref, n_ref = oracle.consensus_general(x, 0.1, 0.01, w, push_from, two_term, d=d)
-    got, r, n = run(binding, x, d, 0.1, 0.01, w, push_from, two_term)
-    assert_parity(got, r, ref, r_ref, d)
-    assert np.all(np.abs(n - n_ref) <= 1e-5 * n_ref + 1e-30)
-    assert np.all(n[n_ref == 0.0] == 0.0)
-    assert_pad_untouched(got, d)
+    got, r, n = run(binding, x, d, 0.1, 0.01, w, push_from, two_term, PATHS[path])
+    check(got, r, n, ref, r_ref, n_ref, d)
+
+
+@pytest.mark.parametrize("wkind,push_from,two_term", [("random", "consensus", True), ("leader", "consensus", False),
+                                                      ("random", "average", True), ("leader", "average", True)])
+@pytest.mark.parametrize("M,d", [(4, 5_000_005), (8, 3_000_017), (12, 2_000_003), (16, 1_500_001)])
+def test_weighted_rounds_with_more_chunks_per_block_than_ring_stages(oracle, M, d, wkind, push_from, two_term):
+    """Vectors long enough that every block wraps its ring several times in the distance pass and
+    refills stages in the update pass, with every flavour of the arithmetic."""
+    _, binding = require_gpu()
+    x = replicas(M, d, seed=M + d % 101)
+    w = weights_for(wkind, M, 3)
+    ref, r_ref, n_ref = oracle.consensus_general(x, 0.1, 0.02, w, push_from, two_term, d=d)
+    got, r, n = run(binding, x, d, 0.1, 0.02, w, push_from, two_term, 3)
+    check(got, r, n, ref, r_ref, n_ref, d)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("weights", [None, [2.0, 2.0, 2.0, 2.0]])
+def test_hard_consensus_with_equal_weights_collapses_onto_the_average(oracle, path, weights):
+    """alpha = 1 (the DDP / hard-consensus case of Algorithm 1) with the push taken from the
+    average: every pulled point IS the average, so no worker has a push direction; the
+    replicas collapse onto x_A and the push distances are exactly zero, whatever lambda is."""
+    _, binding = require_gpu()
+    d = 400_003
+    x = replicas(4, d, seed=71)
+    ref, r_ref, n_ref = oracle.consensus_general(x, 1.0, 0.5, weights, "average", False, d=d)
+    assert np.all(n_ref == 0.0)
+    got, r, n = run(binding, x, d, 1.0, 0.5, weights, "average", False, PATHS[path])
+    assert np.all(n == 0.0)
+    check(got, r, n, ref, r_ref, n_ref, d)
+    spread = np.abs(got[:, :d].astype(np.float64) - got[0, :d]).max()        # all on x_A, to fp32 rounding
+    assert spread <= 4e-9
 
 
 def test_defaults_agree_with_the_plain_round(oracle):

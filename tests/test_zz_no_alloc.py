@@ -10,7 +10,7 @@ with a different worker count and grid), and a worker count above the limit is r
 import numpy as np
 import pytest
 
-from gpu_util import assert_pad_untouched, padded, require_gpu, same_bits, to_dev
+from gpu_util import assert_pad_untouched, assert_parity, padded, require_gpu, same_bits, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -33,7 +33,7 @@ def _both(binding, x_np, d, alpha, lam):
     return xa.cpu().numpy(), na.cpu().numpy(), xb.cpu().numpy(), nb.cpu().numpy()
 
 
-def test_static_scratch_round_matches_workspace_round_twice_in_a_row():
+def test_static_scratch_round_matches_workspace_round_twice_in_a_row(oracle):
     _, binding = require_gpu()
     # call 1: M = 8 on a long vector (full grid); call 2: M = 3 on a short ragged one (small
     # grid), so the second call runs over stale partial sums of the first
@@ -47,6 +47,10 @@ def test_static_scratch_round_matches_workspace_round_twice_in_a_row():
         assert same_bits(xa[:, :d], xb[:, :d]) and same_bits(na, nb)
         assert not same_bits(xb[:, :d], x_np[:, :d])          # the round did run
         assert_pad_untouched(xb, d)
+        # and directly against the CPU oracle, at the tolerances of the parity tests
+        ref, r_ref = oracle.consensus(x_np, alpha, lam, d=d)
+        assert_parity(xb, nb, ref, r_ref, d)
+        assert binding.dppf_static_device_status() == binding.OK
 
 
 def test_static_scratch_round_repeats_and_works_without_norms():
@@ -61,6 +65,45 @@ def test_static_scratch_round_repeats_and_works_without_norms():
         binding.dppf_consensus_static(xb, 0.1, 0.005, d=d)
     torch.cuda.synchronize()
     assert same_bits(xa.cpu().numpy()[:, :d], xb.cpu().numpy()[:, :d])
+
+
+def test_static_scratch_calls_allocate_nothing():
+    """Neither the driver's free-memory figure nor torch's allocator moves across warmed-up calls."""
+    import torch
+    _, binding = require_gpu()
+    d = 1_000_003
+    x = to_dev(_replicas(4, d, 35))
+    norms = torch.zeros(4, device="cuda")
+    binding.dppf_consensus_static(x, 0.1, 0.005, norms_out=norms, d=d)          # first call: set-up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for _ in range(5):
+        binding.dppf_consensus_static(x, 0.1, 0.005, norms_out=norms, d=d)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    assert binding.dppf_static_device_status() == binding.OK
+
+
+def test_static_scratch_status_word_reports_a_give_up():
+    """The status word of the built-in scratch is readable without a workspace pointer: a wait
+    that gives up in the staged kernel (poll budget 0, see test_gpu_timeouts.py) shows up there."""
+    _, binding = require_gpu()
+    d = 1_000_003
+    x_np = _replicas(4, d, 36)
+    x = to_dev(x_np)
+    try:
+        binding.debug_set_poll_limits(0, -1)
+        binding.dppf_consensus_static(x, 0.1, 0.005, d=d)
+        status = binding.dppf_static_device_status()
+    finally:
+        binding.debug_set_poll_limits(-1, -1)
+    assert status == binding.ERR_TIMEOUT
+    assert same_bits(x.cpu().numpy()[:, :d], x_np[:, :d])
+    binding.dppf_consensus_static(x, 0.1, 0.005, d=d)
+    assert binding.dppf_static_device_status() == binding.OK
 
 
 def test_static_scratch_round_refuses_too_many_workers_and_bad_layout():
