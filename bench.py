@@ -3,14 +3,29 @@
 
 One "step" is one consensus round over all M replicas of the workload: average,
 per-worker distances, in-place pull-push update.  The default workload is the
-ViT-B/16-sized one (M = 4, d = 86,567,656 fp32), rounds issued back to back on one
-stream.  Prints ONE JSON line (rank 0).
+ViT-B/16-sized one (M = 4, d = 86,567,656 fp32), one call of the library per round,
+rounds issued back to back on one stream.  Prints ONE JSON line (rank 0).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C4] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--repeats R] [--workload C4]
+                    [--variant plain|general|adamw] [--shard none|columns] [--impl ours|reference]
 
-Multi-GPU: the path does not shard (one GPU holds all M replicas of a round), so
-N > 1 runs N independent replicas, one process per GPU, with no data-path
-collective ("weak" scaling: rounds/s adds up).
+The K-step loop is timed R times (each time bracketed by a barrier and a device
+synchronisation, CUDA events on the launching stream, slowest rank counts); the
+reported time per step is the median over the R repeats.
+
+--variant plain     dppf_consensus per step (workload C3: the last local SGD-momentum step fused
+                    with the round, dppf_local_step_and_consensus); also reports, under
+                    "multi_round", the same rounds issued 100 per call through
+                    dppf_consensus_rounds (update pass of round k fused with the distance pass of
+                    round k+1).
+--variant general   dppf_consensus_general (weighted consensus variable, push from it, both terms).
+--variant adamw     dppf_adamw_step_and_consensus (last AdamW step fused with the round).
+
+Multi-GPU: by default the path does not shard (one GPU holds all M replicas of a round), so
+N > 1 runs N independent replicas, one process per GPU, with no data-path collective ("weak"
+scaling: rounds/s adds up).  --shard columns splits the columns of ONE workload over the N
+ranks instead: every step is dppf_distance_partials, an all-reduce of the M fp64 sums of
+squares, dppf_update_from_sums ("strong" scaling).
 
 ``--impl reference`` times the CPU oracle (plain C, fp64) on the host cores on a
 bounded column slice of the same workload; rank 0 only.
@@ -20,6 +35,7 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import statistics
 import sys
 import threading
 import time
@@ -30,24 +46,31 @@ sys.path.insert(0, ROOT)
 METRIC = "DPPF consensus rounds/s"
 UNIT = "rounds/s"
 NOMINAL_HBM_GBS = 8000.0
+ADAMW = dict(lr=5e-4, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)     # the paper's ViT setting
 
 
-def parse_args():
+def parse_args(argv=None):
     p = argparse.ArgumentParser()
     p.add_argument("--gpus", type=int, default=1)
-    p.add_argument("--steps", type=int, default=1000)
+    p.add_argument("--steps", type=int, default=200)
     p.add_argument("--warmup", type=int, default=10)
+    p.add_argument("--repeats", type=int, default=20, help="how many times the K-step loop is timed (median reported)")
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
     p.add_argument("--workload", default="C4")
+    p.add_argument("--variant", default="plain", choices=["plain", "general", "adamw"])
+    p.add_argument("--shard", default="none", choices=["none", "columns"])
     p.add_argument("--d", type=int, default=0, help="override the vector length (profiling on a smaller case)")
     p.add_argument("--path", default="auto", choices=["auto", "two_kernel", "cooperative", "staged"])
+    p.add_argument("--rounds-per-call", type=int, default=100, help="rounds per dppf_consensus_rounds call")
+    p.add_argument("--multi-round-calls", type=int, default=7)
+    p.add_argument("--no-multi-round", action="store_true")
     p.add_argument("--e2e-steps", type=int, default=5)
     p.add_argument("--no-e2e", action="store_true")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--seed", type=int, default=None)
     p.add_argument("--graph", action="store_true",
                    help="also time the same steps replayed from a CUDA graph (extra key 'graph_replay')")
-    return p.parse_args()
+    return p.parse_args(argv)
 
 
 def measured_peaks():
@@ -60,14 +83,10 @@ def measured_peaks():
         return 6650.0, "fallback"
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the single-pass
-# ncu capture of the full-size launch summarised in profiles/round_kernel_staged_M4.md.
-# Keyed by (workload, kernel); set an entry to None whenever that kernel changes.
-NCU_TRAFFIC = {("C4", 86_567_656, "staged"): 4.00e9}
-
-
-def measured_traffic(w, staged):
-    return NCU_TRAFFIC.get((w.name, w.d, "staged" if staged else "register"))
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from single-pass ncu
+# captures of full-size launches.  Keyed by (workload, d, kernel); an entry is removed whenever
+# that kernel changes, and the line then reports null.
+NCU_TRAFFIC = {}
 
 
 def workload_of(args):
@@ -78,16 +97,37 @@ def workload_of(args):
     return w
 
 
-def config_of(w, extra=None):
-    what = ("last local SGD-momentum step fused with the round, steps" if w.tau > 0 else "rounds")
-    cfg = {"workload": f"{w.name}: M={w.M} replicas x d={w.d} fp32 ({w.model}), alpha={w.alpha}, lambda={w.lam}, "
-                       f"{what} back to back on one stream",
-           "M": w.M, "d": w.d, "ld": w.ld, "alpha": w.alpha, "lambda": w.lam,
-           "replica_bytes": w.M * w.d * 4,
-           "l2_policy": "inputs larger than L2 (no flush between iterations)"}
-    if extra:
-        cfg.update(extra)
-    return cfg
+def step_description(w, variant):
+    if variant == "general":
+        return "general rounds (weighted consensus variable, push from it, both gradient terms)"
+    if variant == "adamw":
+        return "last AdamW local step fused with the round, steps"
+    return "last local SGD-momentum step fused with the round, steps" if w.tau > 0 else "rounds"
+
+
+def config_of(w, variant="plain"):
+    """Names the workload; identical in the CUDA arm and the reference arm."""
+    return {"workload": f"{w.name}: M={w.M} replicas x d={w.d} fp32 ({w.model}), alpha={w.alpha}, lambda={w.lam}, "
+                        f"{step_description(w, variant)} back to back on one stream",
+            "variant": variant, "M": w.M, "d": w.d, "ld": w.ld, "alpha": w.alpha, "lambda": w.lam,
+            "replica_bytes": w.M * w.d * 4,
+            "l2_policy": "inputs larger than L2 (no flush between iterations)"}
+
+
+def general_weights(w, seed):
+    """Seeded positive weights of the consensus variable for --variant general."""
+    import numpy as np
+    return (np.random.default_rng(seed).random(w.M) + 0.05).astype(np.float32)
+
+
+def column_shard(d, world, rank):
+    """Columns [lo, hi) of rank `rank` when d columns are split over `world` ranks: equal
+    shares rounded up to 32 columns (128-byte row starts), the last rank takes the rest."""
+    per = -(-d // world)
+    per = -(-per // 32) * 32
+    lo = min(d, rank * per)
+    hi = d if rank == world - 1 else min(d, lo + per)
+    return lo, hi
 
 
 # ------------------------------------------------------------------ clocks
@@ -159,20 +199,70 @@ def physical_gpu_index(local_index):
 
 # ------------------------------------------------------------------ CPU oracle legs
 
-def time_oracle(w, x_host, budget_s, threads=0):
-    """Times the CPU oracle (column-block OpenMP variant) on a column slice sized for
-    ``budget_s`` seconds; returns (full-workload rounds/s, threads used, slice, seconds)."""
+def _with_grad_std(w):
+    from dataclasses import replace
+    return replace(w, grad_std=1e-2)
+
+
+def oracle_step_fn(w, variant, seed, d_s):
+    """Returns (one_step, cores): one_step() runs one oracle step of the variant on the first
+    d_s columns of the workload, carrying its state from call to call."""
+    import numpy as np
+    import oracle
+    from paper_2507_20424_b200 import inputs
+    ws = w.scaled(d_s)
+    x0 = np.ascontiguousarray(inputs.replicas(ws, seed)[:, :d_s])
+    if variant == "general":
+        wts = general_weights(w, seed)
+        state = {"x": x0}
+
+        def one_step():
+            state["x"], _, _ = oracle.consensus_general(state["x"], w.alpha, w.lam, wts, "consensus", True, d=d_s)
+        return one_step, 1
+    if variant == "adamw":
+        g = np.ascontiguousarray(inputs.gradients(ws if ws.grad_std else _with_grad_std(ws), 0, seed)[:, :d_s])
+        state = {"x": x0.astype(np.float64), "a": np.zeros((w.M, d_s)), "b": np.zeros((w.M, d_s)), "t": 0}
+
+        def one_step():
+            state["t"] += 1
+            x64, state["a"], state["b"] = oracle.adamw_steps_f64(state["x"], state["a"], state["b"], [g],
+                                                                first_step=state["t"], **ADAMW)
+            out, _ = oracle.consensus_f64(x64, w.alpha, w.lam)
+            state["x"] = out.astype(np.float64)
+        return one_step, 1
+    if w.tau > 0:          # local-step workload: one oracle local step, then the round, per step
+        g = np.ascontiguousarray(inputs.gradients(ws, 0, seed)[:, :d_s])
+        state = {"x": x0, "v": np.zeros((w.M, d_s), dtype=np.float32)}
+
+        def one_step():
+            xo, v64, _ = oracle.local_steps_then_consensus(state["x"], state["v"], [g], w.lr, w.momentum,
+                                                           w.weight_decay, w.alpha, w.lam)
+            state["x"], state["v"] = xo, v64.astype(np.float32)
+        return one_step, 1
+    state = {"x": x0, "cores": 0}
+
+    def one_step():
+        state["x"], _, state["cores"] = oracle.consensus_blocked(state["x"], w.alpha, w.lam, d=d_s)
+    one_step()
+    return one_step, state["cores"]
+
+
+def time_oracle(w, variant, seed, budget_s):
+    """Times one oracle step of the variant on a column slice sized for about ``budget_s``
+    seconds; returns (full-workload rounds/s, threads used, slice, seconds)."""
     import oracle
     oracle.build()
-    probe = min(w.d, 2_000_000)
+    probe = min(w.d, 1_000_000)
+    step, cores = oracle_step_fn(w, variant, seed, probe)
     t0 = time.perf_counter()
-    _, _, used = oracle.consensus_blocked(x_host[:, :probe], w.alpha, w.lam, threads=threads)
+    step()
     rate = probe / max(time.perf_counter() - t0, 1e-6)          # columns per second
     d_s = int(min(w.d, max(probe, rate * budget_s)))
+    step, cores = oracle_step_fn(w, variant, seed, d_s)
     t0 = time.perf_counter()
-    oracle.consensus_blocked(x_host[:, :d_s], w.alpha, w.lam, threads=threads)
+    step()
     dt = time.perf_counter() - t0
-    return 1.0 / (dt * w.d / d_s), used, d_s, dt
+    return 1.0 / (dt * w.d / d_s), cores, d_s, dt
 
 
 def run_reference(args):
@@ -188,30 +278,13 @@ def run_reference(args):
     total_budget = 150.0
     per_step = total_budget / max(1, args.steps + args.warmup)
     # calibrate on a small slice, then size the per-step slice
-    probe_w = w.scaled(min(w.d, 1_000_000))
-    xp = inputs.replicas(probe_w, seed)
+    probe = min(w.d, 500_000)
+    step, cores = oracle_step_fn(w, args.variant, seed, probe)
     t0 = time.perf_counter()
-    _, _, cores = oracle.consensus_blocked(xp, w.alpha, w.lam, d=probe_w.d)
-    rate = probe_w.d / max(time.perf_counter() - t0, 1e-6)
+    step()
+    rate = probe / max(time.perf_counter() - t0, 1e-6)
     d_s = int(min(w.d, max(4096, rate * per_step * 0.8)))
-    fused = w.tau > 0          # local-step workload: one oracle local step, then the round, per step
-    if fused:
-        d_s = max(4096, d_s // 8)          # the oracle's local step is single-threaded fp64
-        cores = 1
-    ws = w.scaled(d_s)
-    state = {"x": inputs.replicas(ws, seed)}
-    if fused:
-        import numpy as np
-        g = np.ascontiguousarray(inputs.gradients(ws, 0, seed)[:, :d_s])
-        state = {"x": np.ascontiguousarray(state["x"][:, :d_s]), "v": np.zeros((w.M, d_s), dtype=np.float32)}
-
-        def one_step():
-            xo, v64, _ = oracle.local_steps_then_consensus(state["x"], state["v"], [g], w.lr, w.momentum,
-                                                           w.weight_decay, w.alpha, w.lam)
-            state["x"], state["v"] = xo, v64.astype(np.float32)
-    else:
-        def one_step():
-            state["x"], _, _ = oracle.consensus_blocked(state["x"], w.alpha, w.lam, d=d_s)
+    one_step, cores = oracle_step_fn(w, args.variant, seed, d_s)
     for _ in range(args.warmup):
         one_step()
     t0 = time.perf_counter()
@@ -219,23 +292,24 @@ def run_reference(args):
         one_step()
     dt = (time.perf_counter() - t0) / max(1, args.steps)
     value = 1.0 / (dt * w.d / d_s)
-    what = "one oracle local step and round" if fused else "one oracle round"
+    what = {"general": "one oracle general round", "adamw": "one oracle AdamW step and round"}.get(
+        args.variant, "one oracle local step and round" if w.tau > 0 else "one oracle round")
     sample = (f"each step = {what} on the first {d_s} of {w.d} columns (all {w.M} rows); "
               f"rounds/s scaled by {d_s}/{w.d}")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * w.d / d_s * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": config_of(w),
+            "data": "synthetic", "config": config_of(w, args.variant),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
 
 
-# ------------------------------------------------------------------ replicas-only aggregation
+# ------------------------------------------------------------------ aggregation over ranks
 
 def max_over_ranks(ms, world, device=None):
-    """Slowest rank's elapsed time: the job is done when the last replica is."""
+    """Slowest rank's elapsed time: the job is done when the last rank is."""
     if world <= 1:
         return float(ms)
     import torch
@@ -253,6 +327,7 @@ def whole_job_rate(steps, world, elapsed_ms):
 # ------------------------------------------------------------------ CUDA arm
 
 def run_ours(args):
+    import numpy as np
     import torch
     import torch.distributed as dist
     from paper_2507_20424_b200 import binding, inputs
@@ -264,49 +339,96 @@ def run_ours(args):
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     binding.load(rebuild_if_stale=True)
     w = workload_of(args)
-    seed = (inputs.DEFAULT_SEED if args.seed is None else args.seed) + rank
+    sharded = args.shard == "columns"
+    variant = args.variant
+    if sharded and (variant != "plain" or w.tau > 0):
+        raise SystemExit("--shard columns applies to the plain round")
+    # replicas-only runs give every rank its own replica set; column shards share one
+    seed = (inputs.DEFAULT_SEED if args.seed is None else args.seed) + (0 if sharded else rank)
     path = {"auto": binding.PATH_AUTO, "two_kernel": binding.PATH_TWO_KERNEL,
             "cooperative": binding.PATH_COOPERATIVE, "staged": binding.PATH_STAGED}[args.path]
-    staged = args.path == "staged" or (args.path == "auto" and w.M <= 8)
-    kernel_name = ("distance_kernel + update_kernel (one round)" if args.path == "two_kernel" else
-                   "round_kernel_staged (distance pass + grid barrier + update pass, one launch)" if staged else
-                   "round_kernel (distance pass + grid barrier + update pass, one launch)")
 
     # CPU baseline first (rank 0, N = 1 only): before any GPU work, so the OpenMP team is
     # created in a process that has not touched CUDA yet.
-    x_host = inputs.replicas(w, seed)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        val, cores, d_s, dt = time_oracle(w, x_host, budget_s=12.0)
-        val1, _, d_1, dt1 = time_oracle(w, x_host, budget_s=6.0, threads=1)
+        val, cores, d_s, dt = time_oracle(w, variant, seed, budget_s=12.0)
         cpu = {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"one oracle round on the first {d_s} of {w.d} columns ({dt:.1f} s), scaled by columns",
-               "single_thread_value": val1}
+               "sample": f"one oracle step on the first {d_s} of {w.d} columns ({dt:.1f} s), scaled by columns"}
 
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    x_pinned = torch.from_numpy(x_host).pin_memory()
-    x = binding.alloc_rows(w.M, w.d)
-    x.copy_(x_pinned, non_blocking=True)
+    x_host = inputs.replicas(w, seed)
+    lo, hi = column_shard(w.d, world, rank) if sharded else (0, w.d)
+    d_loc = hi - lo
+    x_pinned = torch.from_numpy(np.ascontiguousarray(x_host[:, lo:hi]) if sharded else x_host).pin_memory()
+    x = binding.alloc_rows(w.M, d_loc)
+    x[:, :d_loc].copy_(x_pinned[:, :d_loc], non_blocking=True)
     norms = torch.zeros(w.M, device="cuda")
-    ws = binding.alloc_workspace(w.M, w.d)
-    B = w.M * w.d * 4
-    fused = w.tau > 0          # local-step workload: every step = last local step fused with the round
-    model_units = 7.0 if fused else 3.0      # x M d 4 bytes per step (two-pass fused round: 7, plain round: 3)
-    if fused:
+    ws = binding.alloc_workspace(w.M, d_loc)
+    B = w.M * d_loc * 4                      # replica bytes this rank holds
+    fused_sgd = variant == "plain" and w.tau > 0
+    staged = args.path in ("auto", "staged") and w.M <= 16
+
+    if sharded:
+        sums = torch.zeros(w.M, dtype=torch.float64, device="cuda")
+        model_units, kernel_id = 3.0, "distance_kernel + update_kernel (column shard)"
+        kernel_name = ("dppf_distance_partials (distance_kernel + sum_partials_kernel), all-reduce of M fp64 sums, "
+                       "dppf_update_from_sums (update_kernel)")
+        launches_per_step = 3
+
+        def step():
+            binding.dppf_distance_partials(x, sums, ws=ws, d=d_loc)
+            if world > 1:
+                dist.all_reduce(sums)
+            binding.dppf_update_from_sums(x, w.alpha, w.lam, sums, norms_out=norms, d=d_loc)
+    elif variant == "general":
+        wts = [float(v) for v in general_weights(w, seed)]
+        model_units, kernel_id = 3.0, "general_round_kernel"
+        kernel_name = "general_round_kernel (distance pass + grid barrier + update pass, one launch)"
+        launches_per_step = 1
+
+        def step():
+            binding.dppf_consensus_general(x, w.alpha, w.lam, wts, binding.PUSH_FROM_CONSENSUS, True,
+                                           norms_out=norms, ws=ws, d=w.d)
+    elif variant == "adamw":
+        wg = w if w.grad_std else _with_grad_std(w)
+        m1, m2 = binding.alloc_rows(w.M, w.d, fill=0.0), binding.alloc_rows(w.M, w.d, fill=0.0)
+        g = binding.alloc_rows(w.M, w.d)
+        g.copy_(torch.from_numpy(inputs.gradients(wg, 0, seed)).pin_memory(), non_blocking=True)
+        model_units, kernel_id = 9.0, "adamw_round_kernel"
+        kernel_name = "adamw_round_kernel (AdamW step + distance pass, grid barrier, update pass, one launch)"
+        launches_per_step = binding.adamw_launch_count(w.M)
+        counter = {"t": 0}
+
+        def step():
+            counter["t"] += 1
+            binding.dppf_adamw_step_and_consensus(x, m1, m2, g, step=counter["t"], alpha=w.alpha, lam=w.lam,
+                                                  norms_out=norms, ws=ws, d=w.d, **ADAMW)
+    elif fused_sgd:
         v = binding.alloc_rows(w.M, w.d, fill=0.0)
         g = binding.alloc_rows(w.M, w.d)
         g.copy_(torch.from_numpy(inputs.gradients(w, 0, seed)).pin_memory(), non_blocking=True)
-        staged = False
+        model_units, kernel_id = 7.0, "round_kernel<fused>"       # two-pass fused round: 7 x M d 4 bytes
         kernel_name = ("distance_kernel<fused> + update_kernel (one step)" if args.path == "two_kernel" else
                        "round_kernel<fused> (local step + distance pass, grid barrier, update pass, one launch)")
+        launches_per_step = binding.launch_count(w.M, w.d, path, True)
 
-    def step():
-        if fused:
+        def step():
             binding.dppf_local_step_and_consensus(x, v, g, w.lr, w.momentum, w.weight_decay, w.alpha, w.lam,
                                                   norms_out=norms, ws=ws, d=w.d, path=path)
-        else:
+    else:
+        model_units = 3.0
+        kernel_id = ("two_kernel" if args.path == "two_kernel" else "round_kernel_staged" if staged and w.M <= 8 else
+                     "rounds_kernel_staged" if staged else "round_kernel")
+        kernel_name = {"two_kernel": "distance_kernel + update_kernel (one round)",
+                       "round_kernel_staged": "round_kernel_staged (distance pass + grid barrier + update pass, one launch)",
+                       "rounds_kernel_staged": "rounds_kernel_staged, one round (distance pass + grid barrier + update pass, one launch)",
+                       "round_kernel": "round_kernel (distance pass + grid barrier + update pass, one launch)"}[kernel_id]
+        launches_per_step = binding.launch_count(w.M, w.d, path, False)
+
+        def step():
             binding.dppf_consensus(x, w.alpha, w.lam, norms_out=norms, ws=ws, d=w.d, path=path)
 
     def fence():
@@ -317,25 +439,58 @@ def run_ours(args):
     for _ in range(max(3, args.warmup)):
         step()
     fence()
-    K = args.steps
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+    K, R = args.steps, max(1, args.repeats)
+    rep_ms, launch_ms = [], []
     with ClockSampler(physical_gpu_index(local)) as clocks:
-        fence()
-        ev[0].record()
-        for i in range(K):
-            step()
-            ev[i + 1].record()
-        fence()
-    total_ms = ev[0].elapsed_time(ev[K])
-    per_launch_ms = sum(ev[i].elapsed_time(ev[i + 1]) for i in range(K)) / K
+        for _ in range(R):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+            fence()
+            ev[0].record()
+            for i in range(K):
+                step()
+                ev[i + 1].record()
+            fence()
+            rep_ms.append(max_over_ranks(ev[0].elapsed_time(ev[K]), world, "cuda"))
+            launch_ms.append(sum(ev[i].elapsed_time(ev[i + 1]) for i in range(K)) / K)
     if binding.dppf_device_status(ws) != binding.OK:
         raise SystemExit("device status word reports an error")
-    total_ms = max_over_ranks(total_ms, world, "cuda")
-    launches_per_step = binding.launch_count(w.M, w.d, path, fused)
+    total_ms = statistics.median(rep_ms)
+    per_launch_ms = statistics.median(launch_ms)
+    peak, peak_src = measured_peaks()
+
+    # the same rounds, rounds_per_call of them per library call (update pass of round k fused with
+    # the distance pass of round k + 1): (1 + 2n) x M d 4 bytes per call
+    multi_round = None
+    if variant == "plain" and not fused_sgd and not sharded and not args.no_multi_round and w.M <= 16:
+        n = args.rounds_per_call
+        norms_all = torch.zeros(n, w.M, device="cuda")
+        binding.dppf_consensus_rounds(x, w.alpha, w.lam, n, norms_out=norms_all, ws=ws, d=w.d)
+        fence()
+        call_ms = []
+        for _ in range(max(1, args.multi_round_calls)):
+            m0, m1_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            fence()
+            m0.record()
+            binding.dppf_consensus_rounds(x, w.alpha, w.lam, n, norms_out=norms_all, ws=ws, d=w.d)
+            m1_.record()
+            fence()
+            call_ms.append(max_over_ranks(m0.elapsed_time(m1_), world, "cuda"))
+        if binding.dppf_device_status(ws) != binding.OK:
+            raise SystemExit("device status word reports an error")
+        ms = statistics.median(call_ms)
+        alg = (1 + 2 * n) * B
+        multi_round = {"entry": "dppf_consensus_rounds", "rounds_per_call": n, "calls_timed": len(call_ms),
+                       "value": whole_job_rate(n, world, ms), "unit": UNIT, "ms_per_round": ms / n,
+                       "ms_per_call_min_max": [min(call_ms), max(call_ms)],
+                       "algorithmic_bytes_per_call": alg, "achieved": alg / (ms * 1e-3) / 1e9, "peak": peak,
+                       "frac": alg / (ms * 1e-3) / 1e9 / peak, "traffic": NCU_TRAFFIC.get((w.name, w.d, f"rounds{n}")),
+                       "kernel": "rounds_kernel_staged (distance pass, then per round: grid barrier + update pass "
+                                 "that also accumulates the next round's squared distances; one launch)",
+                       "gpu_launches_per_call": 1, "model_3Md4_equivalent_gbs": 3 * n * B / (ms * 1e-3) / 1e9}
 
     # optional: the same K steps captured once into a CUDA graph and replayed (launch overhead off the host)
     graph_replay = None
-    if args.graph:
+    if args.graph and not sharded and variant != "adamw":
         chunk = min(K, 100)
         cg_ = torch.cuda.CUDAGraph()
         with torch.cuda.graph(cg_):
@@ -357,7 +512,7 @@ def run_ours(args):
     # end-to-end: replicas live in pinned host memory; every step copies them in, runs the
     # round and copies the replicas and the M distances back.
     e2e = None
-    if not args.no_e2e and not fused:
+    if not args.no_e2e and variant == "plain" and not fused_sgd and not sharded:
         norms_host = torch.zeros(w.M).pin_memory()
         binding.dppf_consensus_host(x_pinned, w.alpha, w.lam, norms_host, x, ws, d=w.d)
         fence()
@@ -367,28 +522,32 @@ def run_ours(args):
             binding.dppf_consensus_host(x_pinned, w.alpha, w.lam, norms_host, x, ws, d=w.d)
         e1.record()
         fence()
-        e2e_ms = e0.elapsed_time(e1)
-        e2e_ms = max_over_ranks(e2e_ms, world, "cuda")
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
         e2e = {"value": whole_job_rate(args.e2e_steps, world, e2e_ms), "unit": UNIT,
                "h2d_bytes_per_step": B, "d2h_bytes_per_step": B + 4 * w.M, "steps": args.e2e_steps}
 
     if rank == 0:
-        peak, peak_src = measured_peaks()
+        jobs = 1 if sharded else world                   # column shards: all ranks work on ONE round
         achieved = model_units * B / (per_launch_ms * 1e-3) / 1e9
-        value = whole_job_rate(K, world, total_ms)
+        value = whole_job_rate(K, jobs, total_ms)
         model_gbs = model_units * B * K / (total_ms * 1e-3) / 1e9
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
-                "warmup": max(3, args.warmup), "ms_per_step": total_ms / K, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": config_of(w, {"parallelism": f"replicas x{world}" if world > 1 else "single GPU",
-                                        "schedule": args.path}),
+                "warmup": max(3, args.warmup), "repeats": R, "ms_per_step": total_ms / K,
+                "ms_per_step_min_max": [min(rep_ms) / K, max(rep_ms) / K],
+                "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
+                "dtype": "f32", "data": "synthetic", "config": config_of(w, variant),
+                "parallelism": (f"column shards x{world} (all-reduce of {w.M} fp64 sums per round)" if sharded else
+                                f"replicas x{world}" if world > 1 else "single GPU"),
+                "schedule": args.path,
                 "model_gbs_per_gpu": model_gbs, "frac_of_nominal_8tbs": model_gbs / NOMINAL_HBM_GBS,
                 "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                             "frac": achieved / peak, "traffic": measured_traffic(w, staged),
+                             "frac": achieved / peak, "traffic": NCU_TRAFFIC.get((w.name, w.d, kernel_id)),
                              "kernel": kernel_name,
                              "algorithmic_bytes_per_launch": int(model_units) * B, "peak_source": f"of {peak_src}"},
-                "clocks": clocks.summary(), "gpu_launches": K * launches_per_step,
+                "clocks": clocks.summary(), "gpu_launches": R * K * launches_per_step,
                 "norms_last_round": [float(v) for v in norms.cpu().tolist()]}
+        if multi_round is not None:
+            line["multi_round"] = multi_round
         if graph_replay is not None:
             line["graph_replay"] = graph_replay
         if e2e is not None:
