@@ -34,97 +34,104 @@ struct GeneralArgs {
     int grid_a;                  // two-launch schedule: blocks of the distance launch
 };
 
+// The per-column arithmetic is written once for fp32 and for packed fp32x2: on sm_100 one
+// add/mul/fma instruction handles two columns (float2), which halves the floating-point
+// instruction count of this arithmetic-heavy round; each lane is rounded exactly like the scalar
+// operation, so both forms give the same bits.
+__device__ __forceinline__ float vsplat(float s, float) { return s; }
+__device__ __forceinline__ float2 vsplat(float s, float2) { return make_float2(s, s); }
+__device__ __forceinline__ float vadd(float a, float b) { return __fadd_rn(a, b); }
+__device__ __forceinline__ float2 vadd(float2 a, float2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ float vsub(float a, float b) { return __fsub_rn(a, b); }
+__device__ __forceinline__ float2 vsub(float2 a, float2 b) { return __fadd2_rn(a, make_float2(-b.x, -b.y)); }
+__device__ __forceinline__ float vmul(float a, float b) { return __fmul_rn(a, b); }
+__device__ __forceinline__ float2 vmul(float2 a, float2 b) { return __fmul2_rn(a, b); }
+__device__ __forceinline__ float vfma(float a, float b, float c) { return __fmaf_rn(a, b, c); }
+__device__ __forceinline__ float2 vfma(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+
 template <int M>
 struct GeneralColumn {
-    // one column: xs[m] in; adds the two squared distances per worker
-    static __device__ __forceinline__ void distances(const float (&xs)[M], const GeneralArgs &a, float (&pr)[M],
-                                                     float (&pn)[M]) {
-        float e[M], ea = 0.f, ec = 0.f;
-        e[0] = 0.f;
+    // one column (V = float) or two (V = float2): xs[m] in; adds the two squared distances per worker
+    template <typename V>
+    static __device__ __forceinline__ void distances(const V (&xs)[M], const GeneralArgs &a, V (&pr)[M], V (&pn)[M]) {
+        const V zero = vsplat(0.f, V()), alpha = vsplat(a.alpha, V());
+        V e[M], ea = zero, ec = zero;
+        e[0] = zero;
 #pragma unroll
         for (int m = 1; m < M; ++m) {
-            e[m] = __fsub_rn(xs[m], xs[0]);
-            ea = __fadd_rn(ea, e[m]);
-            ec = __fmaf_rn(a.wn[m], e[m], ec);
+            e[m] = vsub(xs[m], xs[0]);
+            ea = vadd(ea, e[m]);
+            ec = vfma(vsplat(a.wn[m], V()), e[m], ec);
         }
-        ea = __fmul_rn(ea, 1.0f / (float)M);
+        ea = vmul(ea, vsplat(1.0f / (float)M, V()));
         if (a.uniform) ec = ea;                           // equal weights: the consensus variable IS the average
-        const float p = a.push_from_c ? ec : ea;
+        const V p = a.push_from_c ? ec : ea;
 #pragma unroll
         for (int m = 0; m < M; ++m) {
-            const float dev = __fsub_rn(e[m], ea);
-            pr[m] = __fmaf_rn(dev, dev, pr[m]);
-            const float dy = __fmaf_rn(a.alpha, __fsub_rn(ec, e[m]), __fsub_rn(e[m], p));
-            pn[m] = __fmaf_rn(dy, dy, pn[m]);
+            const V dev = vsub(e[m], ea);
+            pr[m] = vfma(dev, dev, pr[m]);
+            const V dy = vfma(alpha, vsub(ec, e[m]), vsub(e[m], p));
+            pn[m] = vfma(dy, dy, pn[m]);
         }
     }
-    // one column: xs[m] in, updated replicas out; g[m] = lambda / ||y_m - P|| (0: no direction)
-    static __device__ __forceinline__ void update(float (&xs)[M], const GeneralArgs &a, const float *g) {
-        float e[M], ea = 0.f, ec = 0.f;
-        e[0] = 0.f;
+    // one or two columns: xs[m] in, updated replicas out; g[m] = lambda / ||y_m - P|| (0: no direction)
+    template <typename V>
+    static __device__ __forceinline__ void update(V (&xs)[M], const GeneralArgs &a, const float *g) {
+        const V zero = vsplat(0.f, V()), alpha = vsplat(a.alpha, V());
+        V e[M], ea = zero, ec = zero;
+        e[0] = zero;
 #pragma unroll
         for (int m = 1; m < M; ++m) {
-            e[m] = __fsub_rn(xs[m], xs[0]);
-            ea = __fadd_rn(ea, e[m]);
-            ec = __fmaf_rn(a.wn[m], e[m], ec);
+            e[m] = vsub(xs[m], xs[0]);
+            ea = vadd(ea, e[m]);
+            ec = vfma(vsplat(a.wn[m], V()), e[m], ec);
         }
-        ea = __fmul_rn(ea, 1.0f / (float)M);
+        ea = vmul(ea, vsplat(1.0f / (float)M, V()));
         if (a.uniform) ec = ea;                           // equal weights: the consensus variable IS the average
-        const float p = a.push_from_c ? ec : ea;
-        float ub = 0.f;                                   // lambda * mean direction
+        const V p = a.push_from_c ? ec : ea;
+        V ub = zero;                                      // lambda * mean direction
         if (a.two_term) {
 #pragma unroll
             for (int m = 0; m < M; ++m) {
-                const float dy = __fmaf_rn(a.alpha, __fsub_rn(ec, e[m]), __fsub_rn(e[m], p));
-                ub = __fmaf_rn(g[m], dy, ub);
+                const V dy = vfma(alpha, vsub(ec, e[m]), vsub(e[m], p));
+                ub = vfma(vsplat(g[m], V()), dy, ub);
             }
-            ub = __fmul_rn(ub, 1.0f / (float)M);
+            ub = vmul(ub, vsplat(1.0f / (float)M, V()));
         }
 #pragma unroll
         for (int m = 0; m < M; ++m) {
-            const float pull = __fsub_rn(ec, e[m]);       // x_C - x_m
-            const float dy = __fmaf_rn(a.alpha, pull, __fsub_rn(e[m], p));
-            const float y = __fmaf_rn(a.alpha, pull, xs[m]);
-            xs[m] = __fsub_rn(__fmaf_rn(g[m], dy, y), ub);
+            const V pull = vsub(ec, e[m]);                // x_C - x_m
+            const V dy = vfma(alpha, pull, vsub(e[m], p));
+            const V y = vfma(alpha, pull, xs[m]);
+            xs[m] = vsub(vfma(vsplat(g[m], V()), dy, y), ub);
         }
     }
 };
 
-// Four columns of all rows at once (one float4 per row), through the per-column routines.
+// Four columns of all rows at once (one float4 per row) as two packed pairs.
 template <int M>
-__device__ __forceinline__ void general_distances4(const float4 (&xv)[M], const GeneralArgs &a, float (&pr)[M],
-                                                   float (&pn)[M]) {
-    float xs[M];
+__device__ __forceinline__ void general_distances4(const float4 (&xv)[M], const GeneralArgs &a, float2 (&pr)[M],
+                                                   float2 (&pn)[M]) {
+    float2 xs[M];
 #pragma unroll
-    for (int m = 0; m < M; ++m) xs[m] = xv[m].x;
+    for (int m = 0; m < M; ++m) xs[m] = make_float2(xv[m].x, xv[m].y);
     GeneralColumn<M>::distances(xs, a, pr, pn);
 #pragma unroll
-    for (int m = 0; m < M; ++m) xs[m] = xv[m].y;
-    GeneralColumn<M>::distances(xs, a, pr, pn);
-#pragma unroll
-    for (int m = 0; m < M; ++m) xs[m] = xv[m].z;
-    GeneralColumn<M>::distances(xs, a, pr, pn);
-#pragma unroll
-    for (int m = 0; m < M; ++m) xs[m] = xv[m].w;
+    for (int m = 0; m < M; ++m) xs[m] = make_float2(xv[m].z, xv[m].w);
     GeneralColumn<M>::distances(xs, a, pr, pn);
 }
 template <int M>
 __device__ __forceinline__ void general_update4(float4 (&xv)[M], const GeneralArgs &a, const float *g) {
-    float xs[M];
+    float2 lo[M], hi[M];
 #pragma unroll
-    for (int m = 0; m < M; ++m) xs[m] = xv[m].x;
-    GeneralColumn<M>::update(xs, a, g);
+    for (int m = 0; m < M; ++m) {
+        lo[m] = make_float2(xv[m].x, xv[m].y);
+        hi[m] = make_float2(xv[m].z, xv[m].w);
+    }
+    GeneralColumn<M>::update(lo, a, g);
+    GeneralColumn<M>::update(hi, a, g);
 #pragma unroll
-    for (int m = 0; m < M; ++m) { xv[m].x = xs[m]; xs[m] = xv[m].y; }
-    GeneralColumn<M>::update(xs, a, g);
-#pragma unroll
-    for (int m = 0; m < M; ++m) { xv[m].y = xs[m]; xs[m] = xv[m].z; }
-    GeneralColumn<M>::update(xs, a, g);
-#pragma unroll
-    for (int m = 0; m < M; ++m) { xv[m].z = xs[m]; xs[m] = xv[m].w; }
-    GeneralColumn<M>::update(xs, a, g);
-#pragma unroll
-    for (int m = 0; m < M; ++m) xv[m].w = xs[m];
+    for (int m = 0; m < M; ++m) xv[m] = make_float4(lo[m].x, lo[m].y, hi[m].x, hi[m].y);
 }
 
 // Scalar tail columns (d % 4 of them), one thread.
@@ -236,9 +243,9 @@ __global__ void __launch_bounds__(kGeneralThreads, 1) general_round_kernel(const
     for (int m = 0; m < 2 * M; ++m) acc[m] = 0.0;
     int failed = ring_pass<M, StagedShape<M>::kPrefetchA>(ring, a.spin_first, true, 0, [&](float *sb, int k, int) {
         const int cols = ring.cols(k);
-        float pr[M], pn[M];
+        float2 pr[M], pn[M];
 #pragma unroll
-        for (int m = 0; m < M; ++m) pr[m] = pn[m] = 0.f;
+        for (int m = 0; m < M; ++m) pr[m] = pn[m] = make_float2(0.f, 0.f);
         for (int q = tid * 4; q < cols; q += kGeneralThreads * 4) {
             float4 xv[M];
 #pragma unroll
@@ -247,8 +254,8 @@ __global__ void __launch_bounds__(kGeneralThreads, 1) general_round_kernel(const
         }
 #pragma unroll
         for (int m = 0; m < M; ++m) {
-            acc[m] += (double)pr[m];
-            acc[M + m] += (double)pn[m];
+            acc[m] += (double)__fadd_rn(pr[m].x, pr[m].y);
+            acc[M + m] += (double)__fadd_rn(pn[m].x, pn[m].y);
         }
     });
     if (blockIdx.x == 0 && tid == 0 && !failed) general_tail_distances<M>(a, acc);
@@ -282,9 +289,9 @@ template <int M>
 __global__ void __launch_bounds__(Tuning<M>::kThreads, Tuning<M>::kBlocksPerSM) general_distance_kernel(const GeneralArgs a) {
     constexpr int T = Tuning<M>::kThreads;
     __shared__ double s_red[Tuning<M>::kWarps * 2 * M];
-    float pr[M], pn[M];
+    float2 pr[M], pn[M];
 #pragma unroll
-    for (int m = 0; m < M; ++m) pr[m] = pn[m] = 0.f;
+    for (int m = 0; m < M; ++m) pr[m] = pn[m] = make_float2(0.f, 0.f);
     const long long ntiles = (a.nvec + T - 1) / T;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
         const long long j = t * T + threadIdx.x;
@@ -298,8 +305,8 @@ __global__ void __launch_bounds__(Tuning<M>::kThreads, Tuning<M>::kBlocksPerSM) 
     double acc[2 * M];
 #pragma unroll
     for (int m = 0; m < M; ++m) {
-        acc[m] = (double)pr[m];
-        acc[M + m] = (double)pn[m];
+        acc[m] = (double)__fadd_rn(pr[m].x, pr[m].y);
+        acc[M + m] = (double)__fadd_rn(pn[m].x, pn[m].y);
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) general_tail_distances<M>(a, acc);
     general_write_partials<M, Tuning<M>::kWarps>(a, acc, s_red, 0);
