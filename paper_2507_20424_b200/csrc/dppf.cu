@@ -510,7 +510,7 @@ int launch_general_m(const GeneralArgs &a, int path, int dev, cudaStream_t s) {
             int n = 0;
             ready = cudaFuncSetAttribute(general_round_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)smem) == cudaSuccess &&
-                    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, general_round_kernel<M>, kGeneralThreads,
+                    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, general_round_kernel<M>, GeneralShape<M>::kThreads,
                                                                   smem) == cudaSuccess && n >= 1;
             if (ready) g_general_ready[dev][M].store(1, std::memory_order_relaxed);
             else cudaGetLastError();
@@ -523,7 +523,7 @@ int launch_general_m(const GeneralArgs &a, int path, int dev, cudaStream_t s) {
             if (grid < 1) grid = 1;
             void *params[] = {&args};
             if (cudaLaunchCooperativeKernel((const void *)general_round_kernel<M>, dim3((unsigned)grid),
-                                            dim3(kGeneralThreads), params, smem, s) == cudaSuccess)
+                                            dim3(GeneralShape<M>::kThreads), params, smem, s) == cudaSuccess)
                 return DPPF_OK;
             cudaGetLastError();                         // refused (blocks cannot all be resident now): two launches
         }

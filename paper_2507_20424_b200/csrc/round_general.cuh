@@ -16,8 +16,17 @@ namespace {
 // is a per-column register sum, so the second term needs no extra vector or pass.
 // Everything is expressed relative to row 0 (e_m = x_m - x_0), like the shifted mean.
 
-constexpr int kGeneralThreads = 256;   // 384/512/768 threads measured slower (registers)
-constexpr int kGeneralWarps = kGeneralThreads / 32;
+// Threads per block of the cooperative kernel: this round is arithmetic-heavy, so a chunk's float4
+// columns should split evenly over the threads (M = 8: 1280 columns = 320 float4 = 320 threads,
+// not 256 + a quarter-filled second sweep), within the register budget of the worker count.
+template <int M>
+struct GeneralShape {
+    static constexpr int kVecs = StagedShape<M>::kChunk / 4;
+    static constexpr int kMaxThreads = (M <= 4) ? 256 : (M <= 8) ? 384 : 256;
+    static constexpr int kSweeps = (kVecs + kMaxThreads - 1) / kMaxThreads;
+    static constexpr int kThreads = (((kVecs + kSweeps - 1) / kSweeps) + 31) / 32 * 32;
+    static constexpr int kWarps = kThreads / 32;
+};
 
 struct GeneralArgs {
     float *x;
@@ -225,12 +234,12 @@ __device__ __forceinline__ bool general_finalise(const GeneralArgs &a, int nbloc
 
 // One cooperative launch: staged distance pass, grid barrier, staged update pass in reverse.
 template <int M>
-__global__ void __launch_bounds__(kGeneralThreads, 1) general_round_kernel(const GeneralArgs a) {
+__global__ void __launch_bounds__(GeneralShape<M>::kThreads, 1) general_round_kernel(const GeneralArgs a) {
     constexpr int CH = StagedShape<M>::kChunk;
     constexpr int kStages = StagedShape<M>::kStages;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ unsigned long long full[kStages];
-    __shared__ double s_red[kGeneralWarps * 2 * M];
+    __shared__ double s_red[GeneralShape<M>::kWarps * 2 * M];
     __shared__ float s_g[M];
     __shared__ int s_flag;
     const int tid = threadIdx.x;
@@ -246,7 +255,7 @@ __global__ void __launch_bounds__(kGeneralThreads, 1) general_round_kernel(const
         float2 pr[M], pn[M];
 #pragma unroll
         for (int m = 0; m < M; ++m) pr[m] = pn[m] = make_float2(0.f, 0.f);
-        for (int q = tid * 4; q < cols; q += kGeneralThreads * 4) {
+        for (int q = tid * 4; q < cols; q += GeneralShape<M>::kThreads * 4) {
             float4 xv[M];
 #pragma unroll
             for (int m = 0; m < M; ++m) xv[m] = *reinterpret_cast<const float4 *>(sb + m * CH + q);
@@ -259,7 +268,7 @@ __global__ void __launch_bounds__(kGeneralThreads, 1) general_round_kernel(const
         }
     });
     if (blockIdx.x == 0 && tid == 0 && !failed) general_tail_distances<M>(a, acc);
-    general_write_partials<M, kGeneralWarps>(a, acc, s_red, failed);
+    general_write_partials<M, GeneralShape<M>::kWarps>(a, acc, s_red, failed);
     cg::this_grid().sync();
     if (!general_finalise<M>(a, (int)gridDim.x, s_g, &s_flag)) return;
 
@@ -267,7 +276,7 @@ __global__ void __launch_bounds__(kGeneralThreads, 1) general_round_kernel(const
     failed = ring_pass<M, StagedShape<M>::kPrefetchB>(ring, a.spin_later, false, ring.resident(), [&](float *sb, int k, int) {
         const int cols = ring.cols(k);
         float *xg = a.x + ring.col0(k);
-        for (int q = tid * 4; q < cols; q += kGeneralThreads * 4) {
+        for (int q = tid * 4; q < cols; q += GeneralShape<M>::kThreads * 4) {
             float4 xv[M];
 #pragma unroll
             for (int m = 0; m < M; ++m) xv[m] = *reinterpret_cast<const float4 *>(sb + m * CH + q);
