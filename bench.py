@@ -412,9 +412,14 @@ def run_ours(args):
         v = binding.alloc_rows(w.M, w.d, fill=0.0)
         g = binding.alloc_rows(w.M, w.d)
         g.copy_(torch.from_numpy(inputs.gradients(w, 0, seed)).pin_memory(), non_blocking=True)
-        model_units, kernel_id = 7.0, "round_kernel<fused>"       # two-pass fused round: 7 x M d 4 bytes
-        kernel_name = ("distance_kernel<fused> + update_kernel (one step)" if args.path == "two_kernel" else
-                       "round_kernel<fused> (local step + distance pass, grid barrier, update pass, one launch)")
+        model_units = 7.0                                          # two-pass fused round: 7 x M d 4 bytes
+        kernel_id = ("two_kernel<fused>" if args.path == "two_kernel" else
+                     "fused_round_kernel_staged" if staged and w.M <= 8 else "round_kernel<fused>")
+        kernel_name = {"two_kernel<fused>": "distance_kernel<fused> + update_kernel (one step)",
+                       "fused_round_kernel_staged": "fused_round_kernel_staged (local step + distance pass staged through "
+                                                    "shared memory, grid barrier, staged update pass, one launch)",
+                       "round_kernel<fused>": "round_kernel<fused> (local step + distance pass, grid barrier, update "
+                                              "pass, one launch)"}[kernel_id]
         launches_per_step = binding.launch_count(w.M, w.d, path, True)
 
         def step():

@@ -31,8 +31,19 @@
  *   - Zero distance (r_m == 0, e.g. M == 1 or identical replicas): the paper
  *     leaves 0/0 undefined; here no push is applied, the replica is left
  *     bit-for-bit unchanged and r_m = 0 is reported.
- *   - Results are run-to-run reproducible on a given GPU model: the tile-to-block
- *     map is static and every reduction runs in a fixed order (no float atomics).
+ *   - Results are run-to-run reproducible on a given GPU model for a given kernel schedule:
+ *     the tile-to-block map is static and every reduction runs in a fixed order (no float
+ *     atomics).  Different schedules (DPPF_PATH_*) group the sums of squares differently and
+ *     may differ in the last bits of r_m and hence of x.  A call whose cooperative launch the
+ *     runtime refuses falls back to a two-launch schedule (see dppf_consensus_ex); a caller
+ *     that needs bit-identical repeats under such conditions asks for DPPF_PATH_TWO_KERNEL.
+ *   - Accuracy against the definition evaluated in fp64: r_m to 1e-5 relative (fp32 squares
+ *     summed in short fp32 runs, then fp64); every updated element to 1e-6 (1 + |x|) for
+ *     replicas that lie close together compared with their magnitude and a push of the order
+ *     of the distances, the regime of trained replicas.  x_m + (x_A - x_m) c_m is formed in fp32
+ *     from x_m and c_m (x_A - x_m), so its error is about one fp32 ulp of the larger of the two
+ *     terms: when the replicas are as far apart as they are large, or lambda / r_m is large
+ *     (a push much longer than the distances), allow 1.5e-7 max(|x_m|, |step|) on top.
  */
 #ifndef DPPF_H
 #define DPPF_H
@@ -196,6 +207,10 @@ int dppf_local_step_and_consensus(float *x, float *v, const float *g, int M, int
                                   float alpha, float lambda, float *norms_out, void *ws,
                                   size_t ws_bytes, void *cuda_stream);
 
+/* With an explicit schedule.  AUTO picks DPPF_PATH_STAGED for M <= 8 (x, v and g streamed
+ * through shared memory in the step-and-distance pass, the plain staged update pass after the
+ * grid barrier) and DPPF_PATH_COOPERATIVE (register kernel) above.  The fused call rewrites x
+ * and v in its first pass already, so after a DPPF_ERR_TIMEOUT status they are partly stepped. */
 int dppf_local_step_and_consensus_ex(float *x, float *v, const float *g, int M, int64_t d,
                                      int64_t ld, float lr, float momentum, float weight_decay,
                                      float alpha, float lambda, float *norms_out, void *ws,

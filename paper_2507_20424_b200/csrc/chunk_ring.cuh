@@ -59,24 +59,27 @@ __device__ __forceinline__ void bulk_load(void *dst_smem, const void *src, unsig
                  ::"r"(smem_addr(dst_smem)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
 
-template <int M>
+// Ring of kStages stages; a stage holds the same chunk of kChunk columns of the M rows of each of
+// kArrays arrays that share one layout (x alone, or x with optimiser state and gradients).
+template <int M, int kArrays = 1, int kChunk = StagedShape<M>::kChunk, int kStages_ = StagedShape<M>::kStages>
 struct ChunkRing {
-    static constexpr int CH = StagedShape<M>::kChunk;
-    static constexpr int kStages = StagedShape<M>::kStages;
-    float *ring;                   // [kStages][M][CH]
+    static constexpr int CH = kChunk;
+    static constexpr int kStages = kStages_;
+    static constexpr int kRows = kArrays * M;          // row copies per stage
+    static constexpr size_t kStageFloats = (size_t)kRows * CH;
+    static constexpr size_t kSmemBytes = (size_t)kStages * kStageFloats * sizeof(float);
+    float *ring;                   // [kStages][kArrays][M][CH]
     unsigned long long *full;      // one mbarrier per stage
-    const float *x;
+    const float *base[kArrays];
     long long ld, d4;              // row stride; columns covered by float4 groups
     int n;                         // chunks of this block; local chunk k = global chunk blockIdx.x + k gridDim.x,
                                    // always staged in ring stage k % kStages
     unsigned phase;                // bit st: parity of the next wait on stage st
 
-    // to be called by all threads of the block, once
-    __device__ __forceinline__ void init(void *smem, unsigned long long *bars, const float *rows, long long ld_,
-                                         long long nvec) {
+    // to be called by all threads of the block, once; set base[] before
+    __device__ __forceinline__ void init(void *smem, unsigned long long *bars, long long ld_, long long nvec) {
         ring = reinterpret_cast<float *>(smem);
         full = bars;
-        x = rows;
         ld = ld_;
         d4 = nvec * 4;
         const long long nchunks = (d4 + CH - 1) / CH;
@@ -94,14 +97,26 @@ struct ChunkRing {
         const long long c0 = col0(k);
         return (int)((d4 - c0 < CH) ? (d4 - c0) : CH);
     }
-    __device__ __forceinline__ float *stage(int st) const { return ring + (size_t)st * M * CH; }
-    // called by all of warp 0: lane 0 announces the bytes, lanes 0..M-1 copy one row each
+    __device__ __forceinline__ float *stage(int st) const { return ring + (size_t)st * kStageFloats; }
+    // called by all of warp 0: lane 0 announces the bytes, then one row copy per lane
     __device__ __forceinline__ void issue(int k, int st) {
         const unsigned bytes = (unsigned)cols(k) * 4u;
         const int lane = threadIdx.x;
-        if (lane == 0) mbar_expect_tx(&full[st], bytes * M);
+        if (lane == 0) mbar_expect_tx(&full[st], bytes * kRows);
         __syncwarp();
-        if (lane < M) bulk_load(ring + ((size_t)st * M + lane) * CH, x + lane * ld + col0(k), bytes, &full[st]);
+        const long long c0 = col0(k);
+#pragma unroll
+        for (int r0 = 0; r0 < kRows; r0 += 32) {
+            const int r = r0 + lane;
+            if (r < kRows) {
+                const int arr = r / M, m = r - arr * M;
+                const float *src = base[0];
+#pragma unroll
+                for (int i = 1; i < kArrays; ++i)
+                    if (arr == i) src = base[i];
+                bulk_load(ring + (size_t)st * kStageFloats + (size_t)r * CH, src + m * ld + c0, bytes, &full[st]);
+            }
+        }
     }
     __device__ __forceinline__ bool wait(int st, int limit) {
         if (mbar_wait_bounded(&full[st], (phase >> st) & 1u, limit)) {
@@ -120,9 +135,9 @@ struct ChunkRing {
 // async proxy later).  `limit` bounds every wait in polls.  If a wait gives up, the block stops
 // the pass, thread 0 waits (full budget) for the copies still in flight, and 1 is returned in
 // every thread; otherwise 0.
-template <int M, int kPrefetch, typename Body>
-__device__ __forceinline__ int ring_pass(ChunkRing<M> &ring, int limit, bool fwd, int resident, Body body) {
-    constexpr int kStages = StagedShape<M>::kStages;
+template <int kPrefetch, typename Ring, typename Body>
+__device__ __forceinline__ int ring_pass(Ring &ring, int limit, bool fwd, int resident, Body body) {
+    constexpr int kStages = Ring::kStages;
     static_assert(kPrefetch >= 1 && kPrefetch < kStages, "prefetch distance must leave a free stage");
     const int tid = threadIdx.x, n = ring.n;
     int failed = 0;

@@ -6,6 +6,7 @@
 //   chunk_ring.cuh      shared-memory chunk ring of the staged kernels (bulk async copies, bounded waits)
 //   round_staged.cuh    staged persistent round kernel, one round per launch
 //   round_multi.cuh     several rounds in one launch (update pass of round k + distances of round k+1)
+//   round_fused_staged.cuh  local step (SGD-momentum or AdamW) + round, rows staged through shared memory
 //   round_general.cuh   general round (weighted consensus variable, push reference, two-term push)
 //   round_generic.cuh   any worker count up to 1024, stand-alone SGD-momentum local step
 //
@@ -37,6 +38,7 @@
 #include "chunk_ring.cuh"
 #include "round_staged.cuh"
 #include "round_multi.cuh"
+#include "round_fused_staged.cuh"
 #include "round_general.cuh"
 #include "round_generic.cuh"
 
@@ -123,12 +125,57 @@ int blocks_per_sm(K kernel, int dev, int M, int kind, int threads, size_t dyn_sm
     return n;
 }
 
+std::atomic<int> g_fused_ready[64][9];
+
+// Staged fused round (M <= 8).  DPPF_ERR_CUDA + *refused when it cannot be launched cooperatively.
+template <int M>
+int launch_fused_staged_m(const RoundArgs &a, int dev, cudaStream_t s, bool *refused) {
+    *refused = true;
+    if constexpr (M <= 8) {
+        using RingA = ChunkRing<M, FusedShape<M>::kArrays, FusedShape<M>::kChunk, FusedShape<M>::kStages>;
+        constexpr size_t smem = RingA::kSmemBytes > StagedShape<M>::kSmemBytes ? RingA::kSmemBytes
+                                                                               : StagedShape<M>::kSmemBytes;
+        const int sms = sm_count(dev);
+        if (sms <= 0 || !coop_supported(dev)) return DPPF_ERR_CUDA;
+        if (g_fused_ready[dev][M].load(std::memory_order_relaxed) == 0) {
+            int n = 0;
+            if (cudaFuncSetAttribute(fused_round_kernel_staged<M>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)smem) != cudaSuccess ||
+                cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fused_round_kernel_staged<M>, kStagedThreads,
+                                                              smem) != cudaSuccess || n < 1) {
+                cudaGetLastError();
+                return DPPF_ERR_CUDA;
+            }
+            g_fused_ready[dev][M].store(1, std::memory_order_relaxed);
+        }
+        const long long nchunks = (a.nvec * 4 + RingA::CH - 1) / RingA::CH;
+        long long grid = sms;
+        if (grid > nchunks) grid = nchunks;
+        if (grid < 1) grid = 1;
+        RoundArgs aa = a;
+        void *params[] = {&aa};
+        if (cudaLaunchCooperativeKernel((const void *)fused_round_kernel_staged<M>, dim3((unsigned)grid),
+                                        dim3(kStagedThreads), params, smem, s) == cudaSuccess) {
+            *refused = false;
+            return DPPF_OK;
+        }
+        cudaGetLastError();
+    }
+    return DPPF_ERR_CUDA;
+}
+
 template <int M>
 int launch_rounds_m(RoundsArgs &a, int path, int dev, cudaStream_t s, bool *refused);
 RoundsArgs one_round_args(const RoundArgs &a);
 
 template <int M>
 int launch_round_m(RoundArgs a, bool fused, int path, int dev, cudaStream_t s) {
+    if (path == DPPF_PATH_STAGED && fused && M <= 8) {
+        bool refused = false;
+        const int rc = launch_fused_staged_m<M>(a, dev, s, &refused);
+        if (rc == DPPF_OK || !refused) return rc;
+        path = DPPF_PATH_COOPERATIVE;
+    }
     if (path == DPPF_PATH_STAGED && !fused && M > 8) {
         // above eight rows the multi-round kernel (row copies issued by one lane each) is the faster
         // staged kernel; a single round is its two-pass special case
@@ -243,9 +290,9 @@ int launch_local_step(float *x, float *v, const float *g, int M, int64_t d, int6
 
 int resolve_path(int path, int M, bool fused) {
     if (M > kMaxTemplateM) return DPPF_PATH_TWO_KERNEL;
-    if (fused && path == DPPF_PATH_STAGED) return DPPF_PATH_COOPERATIVE;   // no staged kernel with the local step
+    if (fused && path == DPPF_PATH_STAGED && M > 8) return DPPF_PATH_COOPERATIVE;   // staged fused kernel: M <= 8
     // one launch per round, rows staged through shared memory
-    if (path == DPPF_PATH_AUTO) return fused ? DPPF_PATH_COOPERATIVE : DPPF_PATH_STAGED;
+    if (path == DPPF_PATH_AUTO) return (fused && M > 8) ? DPPF_PATH_COOPERATIVE : DPPF_PATH_STAGED;
     return path;
 }
 
@@ -976,7 +1023,8 @@ int dppf_adamw_step_and_consensus_ex(float *x, float *exp_avg, float *exp_avg_sq
     a.partials = reinterpret_cast<double *>(static_cast<unsigned char *>(ws) + kHeaderBytes);
     a.norms_stage = reinterpret_cast<float *>(static_cast<unsigned char *>(ws) + norms_stage_offset(M));
     a.M = M;
-    a.spin_first = a.spin_later = kSpinLimit;
+    a.spin_first = g_spin_first.load(std::memory_order_relaxed);
+    a.spin_later = g_spin_later.load(std::memory_order_relaxed);
     if (M == 1) {
         if ((rc = launch_adamw_step(x, p, M, d, ld, dev, s)) != DPPF_OK) return rc;
         zero_norms_kernel<<<1, 32, 0, s>>>(norms_out, a.norms_stage, a.hdr);

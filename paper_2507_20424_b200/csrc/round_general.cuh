@@ -244,13 +244,14 @@ __global__ void __launch_bounds__(GeneralShape<M>::kThreads, 1) general_round_ke
     __shared__ int s_flag;
     const int tid = threadIdx.x;
     ChunkRing<M> ring;
-    ring.init(smem_raw, full, a.x, a.ld, a.nvec);
+    ring.base[0] = a.x;
+    ring.init(smem_raw, full, a.ld, a.nvec);
 
     // ---- distance pass: sum (x_m - x_A)^2 and sum (y_m - P)^2 per worker
     double acc[2 * M];
 #pragma unroll
     for (int m = 0; m < 2 * M; ++m) acc[m] = 0.0;
-    int failed = ring_pass<M, StagedShape<M>::kPrefetchA>(ring, a.spin_first, true, 0, [&](float *sb, int k, int) {
+    int failed = ring_pass<StagedShape<M>::kPrefetchA>(ring, a.spin_first, true, 0, [&](float *sb, int k, int) {
         const int cols = ring.cols(k);
         float2 pr[M], pn[M];
 #pragma unroll
@@ -273,7 +274,7 @@ __global__ void __launch_bounds__(GeneralShape<M>::kThreads, 1) general_round_ke
     if (!general_finalise<M>(a, (int)gridDim.x, s_g, &s_flag)) return;
 
     // ---- update pass, chunks in reverse, newest chunks reused from the ring
-    failed = ring_pass<M, StagedShape<M>::kPrefetchB>(ring, a.spin_later, false, ring.resident(), [&](float *sb, int k, int) {
+    failed = ring_pass<StagedShape<M>::kPrefetchB>(ring, a.spin_later, false, ring.resident(), [&](float *sb, int k, int) {
         const int cols = ring.cols(k);
         float *xg = a.x + ring.col0(k);
         for (int q = tid * 4; q < cols; q += GeneralShape<M>::kThreads * 4) {

@@ -88,7 +88,8 @@ __global__ void __launch_bounds__(kStagedThreads, 1) rounds_kernel_staged(const 
     __shared__ float s_c[M];
     const int tid = threadIdx.x;
     ChunkRing<M> ring;
-    ring.init(smem_raw, full, a.x, a.ld, a.nvec);
+    ring.base[0] = a.x;
+    ring.init(smem_raw, full, a.ld, a.nvec);
     const int n = ring.n;
 
     // tail columns (d % 4 of them) go through the scalar routines, which take the single-round arguments
@@ -105,15 +106,15 @@ __global__ void __launch_bounds__(kStagedThreads, 1) rounds_kernel_staged(const 
         for (int m = 0; m < M; ++m) acc[m] = 0.0;
         int failed;
         if (first) {
-            failed = ring_pass<M, StagedShape<M>::kPrefetchA>(ring, a.spin_first, fwd, 0, [&](float *sb, int k, int) {
+            failed = ring_pass<StagedShape<M>::kPrefetchA>(ring, a.spin_first, fwd, 0, [&](float *sb, int k, int) {
                 chunk_body<M, false>(sb, nullptr, 0, ring.cols(k), s_c, false, true, acc);
             });
         } else if (last) {
-            failed = ring_pass<M, StagedShape<M>::kPrefetchB>(ring, a.spin_later, fwd, ring.resident(), [&](float *sb, int k, int) {
+            failed = ring_pass<StagedShape<M>::kPrefetchB>(ring, a.spin_later, fwd, ring.resident(), [&](float *sb, int k, int) {
                 chunk_body<M, true>(sb, a.x + ring.col0(k), a.ld, ring.cols(k), s_c, false, false, acc);
             });
         } else {
-            failed = ring_pass<M, StagedShape<M>::kPrefetchB>(ring, a.spin_later, fwd, ring.resident(), [&](float *sb, int k, int i) {
+            failed = ring_pass<StagedShape<M>::kPrefetchB>(ring, a.spin_later, fwd, ring.resident(), [&](float *sb, int k, int i) {
                 // chunks this pass handles last are the first of the next pass: keep them current in the ring
                 const bool write_back = i >= n - kStages;
                 chunk_body<M, true>(sb, a.x + ring.col0(k), a.ld, ring.cols(k), s_c, write_back, true, acc);

@@ -94,6 +94,39 @@ def test_give_up_in_an_update_pass_is_reported(oracle, name):
     assert_parity(x.cpu().numpy(), norms.cpu().numpy(), ref, r_ref, d)
 
 
+@pytest.mark.parametrize("limits", [(0, -1), (-1, 0)])
+def test_give_up_in_the_fused_local_step_round_is_reported(oracle, limits):
+    """The staged kernel that fuses the last SGD-momentum step with the round: its first pass
+    already rewrites x and v, so a give-up leaves them partly stepped; what is promised is the
+    status word, rows that stay inside their bounds, and a working library afterwards."""
+    import torch
+    from paper_2507_20424_b200 import inputs
+    _, binding = require_gpu()
+    M, d = 4, 6_000_005
+    w = inputs.WORKLOADS["C3"].scaled(d)
+    x_np, v_np, g_np = inputs.replicas(w), inputs.zeros_like_rows(w), inputs.gradients(w, 0)
+    x_np[:, :d] += inputs.gradients(w, 3)[:, :d]
+    x, v, g = to_dev(x_np), to_dev(v_np), to_dev(g_np)
+    ws = binding.alloc_workspace(M, d)
+    try:
+        binding.debug_set_poll_limits(*limits)
+        binding.dppf_local_step_and_consensus(x, v, g, w.lr, w.momentum, w.weight_decay, w.alpha, w.lam, ws=ws, d=d,
+                                              path=3)
+        status = binding.dppf_device_status(ws)
+    finally:
+        binding.debug_set_poll_limits(-1, -1)
+    assert status == binding.ERR_TIMEOUT
+    assert_pad_untouched(x.cpu().numpy(), d), assert_pad_untouched(v.cpu().numpy(), d)
+    x.copy_(torch.from_numpy(x_np)), v.copy_(torch.from_numpy(v_np))
+    norms = torch.zeros(M, device="cuda")
+    binding.dppf_local_step_and_consensus(x, v, g, w.lr, w.momentum, w.weight_decay, w.alpha, w.lam, norms_out=norms,
+                                          ws=ws, d=d, path=3)
+    assert binding.dppf_device_status(ws) == binding.OK
+    ref, _, r_ref = oracle.local_steps_then_consensus(x_np[:, :d], v_np[:, :d], [g_np[:, :d]], w.lr, w.momentum,
+                                                      w.weight_decay, w.alpha, w.lam)
+    assert_parity(x.cpu().numpy(), norms.cpu().numpy(), ref, r_ref, d)
+
+
 def test_default_budget_is_restored():
     _, binding = require_gpu()
     d = 300_001
