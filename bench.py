@@ -86,7 +86,15 @@ def measured_peaks():
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from single-pass ncu
 # captures of full-size launches.  Keyed by (workload, d, kernel); an entry is removed whenever
 # that kernel changes, and the line then reports null.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    ("C4", 86_567_656, "round_kernel_staged"): 4.008e9,
+    ("C4", 86_567_656, "rounds100"): 264.5e9,
+    ("C2", 26_200_000, "round_kernel_staged"): 2.368e9,
+    ("C5", 44_549_160, "rounds_kernel_staged"): 8.411e9,
+    ("C3", 25_557_032, "fused_round_kernel_staged"): 2.746e9,
+    ("C4", 86_567_656, "general_round_kernel"): 4.007e9,
+    ("C4", 86_567_656, "adamw_round_kernel"): 12.364e9,
+}
 
 
 def workload_of(args):
