@@ -64,7 +64,9 @@ typedef enum {
     DPPF_ERR_TIMEOUT = 5       /* device status only: a bounded wait on an async copy gave up */
 } dppf_status;
 
-/* Largest worker count handled (rows of x). */
+/* Largest worker count handled (rows of x).  The kernels are built for the worker counts the
+ * paper runs (4 and 8) and up to 16: those stream at about the device's copy rate.  Above 16
+ * a simpler kernel family keeps the call correct but reaches only 0.2-0.5 of that rate. */
 #define DPPF_MAX_WORKERS 1024
 
 /* Kernel schedule selector for the *_ex entry points. */
@@ -339,6 +341,15 @@ int dppf_device_status(const void *ws, void *cuda_stream);
  * Always returns DPPF_OK.
  */
 int dppf_debug_set_poll_limits(int first_pass_polls, int later_pass_polls);
+
+/*
+ * Synchronises `cuda_stream` and returns which schedule the last call on this workspace
+ * actually ran (DPPF_PATH_TWO_KERNEL, DPPF_PATH_COOPERATIVE or DPPF_PATH_STAGED): AUTO resolved,
+ * and a fallback taken when the runtime refused a cooperative launch made visible.  Two calls
+ * on the same input give the same bits if they report the same schedule.  Negative if the
+ * stream failed.
+ */
+int dppf_device_schedule(const void *ws, void *cuda_stream);
 
 /* Static, human-readable name of a dppf_status. */
 const char *dppf_status_string(int status);

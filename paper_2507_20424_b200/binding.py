@@ -19,7 +19,7 @@ OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range
 
 EXPORTS = ("dppf_workspace_bytes", "dppf_consensus", "dppf_consensus_ex", "dppf_local_step",
            "dppf_local_step_and_consensus", "dppf_local_step_and_consensus_ex",
-           "dppf_consensus_host", "dppf_device_status", "dppf_status_string", "dppf_launch_count",
+           "dppf_consensus_host", "dppf_device_status", "dppf_device_schedule", "dppf_status_string", "dppf_launch_count",
            "dppf_consensus_static", "dppf_static_device_status", "dppf_consensus_general", "dppf_consensus_general_ex",
            "dppf_distance_partials", "dppf_update_from_sums", "dppf_adamw_step_and_consensus_ex",
            "dppf_consensus_rounds", "dppf_consensus_rounds_ex", "dppf_debug_set_poll_limits",
@@ -60,6 +60,8 @@ def load(rebuild_if_stale: bool = False) -> ctypes.CDLL:
     lib.dppf_local_step_and_consensus_ex.argtypes = [vp, vp, vp, i32, i64, i64, f32, f32, f32, f32, f32, vp, vp, sz, i32, vp]
     lib.dppf_consensus_host.argtypes = [vp, i32, i64, i64, f32, f32, vp, vp, vp, sz, vp]
     lib.dppf_device_status.argtypes = [vp, vp]
+    lib.dppf_device_schedule.argtypes = [vp, vp]
+    lib.dppf_device_schedule.restype = i32
     lib.dppf_lambda_schedule.argtypes = [i32, f32, i64, i64]
     lib.dppf_lambda_schedule.restype = f32
     lib.dppf_lr_cosine.argtypes = [f32, i64, i64]
@@ -102,7 +104,7 @@ def load(rebuild_if_stale: bool = False) -> ctypes.CDLL:
     lib.dppf_status_string.restype = ctypes.c_char_p
     lib.dppf_launch_count.argtypes = [i32, i64, i32, i32]
     for name in ("dppf_consensus", "dppf_consensus_ex", "dppf_local_step", "dppf_local_step_and_consensus",
-                 "dppf_local_step_and_consensus_ex", "dppf_consensus_host", "dppf_device_status",
+                 "dppf_local_step_and_consensus_ex", "dppf_consensus_host", "dppf_device_status", "dppf_device_schedule",
                  "dppf_launch_count"):
         getattr(lib, name).restype = i32
     _lib = lib
@@ -323,6 +325,11 @@ def dppf_round_metrics(norms, alpha, lam):
 
 def dppf_device_status(ws) -> int:
     return int(load().dppf_device_status(ws.data_ptr(), _stream()))
+
+
+def dppf_device_schedule(ws) -> int:
+    """PATH_* of the kernels that ran the last call on this workspace (synchronises the stream)."""
+    return int(load().dppf_device_schedule(ws.data_ptr(), _stream()))
 
 
 def launch_count(M: int, d: int, path=PATH_AUTO, fused=False) -> int:

@@ -125,6 +125,7 @@ __device__ __forceinline__ void adamw_distance_pass(const RoundArgs &a, const Ad
         a.hdr->magic = kMagic;
         a.hdr->grid = (int)gridDim.x;
         a.hdr->M = M;
+        a.hdr->schedule = a.schedule;
     }
 }
 

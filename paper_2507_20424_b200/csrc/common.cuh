@@ -26,6 +26,7 @@ struct WsHeader {
     unsigned magic;   // written by the distance pass, checked by the update pass
     int grid;         // blocks that wrote partials
     int M;
+    int schedule;     // DPPF_PATH_* of the kernels that ran the last call on this workspace
 };
 
 struct RoundArgs {
@@ -40,6 +41,7 @@ struct RoundArgs {
     double *partials; // [grid, M]
     int M;            // runtime copy (generic kernels)
     int spin_first, spin_later;   // staged kernel: mbarrier polls before a wait gives up (distance / update pass)
+    int schedule;                 // DPPF_PATH_* being launched, recorded in the workspace header
 };
 
 // ---------------------------------------------------------------- memory access helpers

@@ -153,6 +153,7 @@ int launch_fused_staged_m(const RoundArgs &a, int dev, cudaStream_t s, bool *ref
         if (grid > nchunks) grid = nchunks;
         if (grid < 1) grid = 1;
         RoundArgs aa = a;
+        aa.schedule = DPPF_PATH_STAGED;
         void *params[] = {&aa};
         if (cudaLaunchCooperativeKernel((const void *)fused_round_kernel_staged<M>, dim3((unsigned)grid),
                                         dim3(kStagedThreads), params, smem, s) == cudaSuccess) {
@@ -200,6 +201,7 @@ int launch_round_m(RoundArgs a, bool fused, int path, int dev, cudaStream_t s) {
             long long grid = sms;                       // one block per SM
             if (grid > nchunks) grid = nchunks;
             if (grid < 1) grid = 1;
+            a.schedule = DPPF_PATH_STAGED;
             void *params[] = {&a};
             if (cudaLaunchCooperativeKernel((const void *)round_kernel_staged<M>, dim3((unsigned)grid),
                                             dim3(kStagedThreads), params, smem, s) == cudaSuccess)
@@ -234,12 +236,14 @@ int launch_round_m(RoundArgs a, bool fused, int path, int dev, cudaStream_t s) {
     if (grid > kMaxBlocksSmallM) grid = kMaxBlocksSmallM;
 
     if (path == DPPF_PATH_COOPERATIVE && coop_supported(dev)) {
+        a.schedule = DPPF_PATH_COOPERATIVE;
         void *params[] = {&a};
         const void *fn = fused ? (const void *)round_kernel<M, true> : (const void *)round_kernel<M, false>;
         if (cudaLaunchCooperativeKernel(fn, dim3((unsigned)grid), dim3(T), params, 0, s) == cudaSuccess)
             return DPPF_OK;
         cudaGetLastError();                             // cooperative launch refused: fall back to two launches
     }
+    a.schedule = DPPF_PATH_TWO_KERNEL;
     if (fused) {
         distance_kernel<M, true><<<(unsigned)grid, T, 0, s>>>(a);
         update_kernel<M, true><<<(unsigned)grid, T, 0, s>>>(a, (int)grid);
@@ -252,6 +256,7 @@ int launch_round_m(RoundArgs a, bool fused, int path, int dev, cudaStream_t s) {
 }
 
 int launch_round_generic(RoundArgs a, bool fused, int dev, cudaStream_t s) {
+    a.schedule = DPPF_PATH_TWO_KERNEL;
     const int sms = sm_count(dev);
     if (sms <= 0) return DPPF_ERR_CUDA;
     long long ntiles = (a.nvec + kThreads - 1) / kThreads;
@@ -331,6 +336,7 @@ int run_round(float *x, float *v, const float *g, int M, int64_t d, int64_t ld, 
     a.M = M;
     a.spin_first = g_spin_first.load(std::memory_order_relaxed);
     a.spin_later = g_spin_later.load(std::memory_order_relaxed);
+    a.schedule = DPPF_PATH_TWO_KERNEL;
 
     if (M == 1) {   // x_A == x_1: distance 0, replica unchanged
         if (fused && (rc = launch_local_step(x, v, g, M, d, ld, lr, mu, wd, dev, s)) != DPPF_OK) return rc;
@@ -479,6 +485,7 @@ int launch_rounds_m(RoundsArgs &a, int path, int dev, cudaStream_t s, bool *refu
     if (sms <= 0) return DPPF_ERR_CUDA;
     if (!coop_supported(dev)) { *refused = true; return DPPF_ERR_CUDA; }
     void *params[] = {&a};
+    a.schedule = (path == DPPF_PATH_STAGED) ? DPPF_PATH_STAGED : DPPF_PATH_COOPERATIVE;
     if (path == DPPF_PATH_STAGED) {
         constexpr size_t smem = StagedShape<M>::kSmemBytes;
         if (g_rounds_ready[dev][M][0].load(std::memory_order_relaxed) == 0) {
@@ -568,6 +575,7 @@ int launch_general_m(const GeneralArgs &a, int path, int dev, cudaStream_t s) {
             if (grid > nchunks) grid = nchunks;
             if (grid > kMaxBlocksSmallM / 2) grid = kMaxBlocksSmallM / 2;
             if (grid < 1) grid = 1;
+            args.schedule = DPPF_PATH_STAGED;
             void *params[] = {&args};
             if (cudaLaunchCooperativeKernel((const void *)general_round_kernel<M>, dim3((unsigned)grid),
                                             dim3(GeneralShape<M>::kThreads), params, smem, s) == cudaSuccess)
@@ -582,6 +590,7 @@ int launch_general_m(const GeneralArgs &a, int path, int dev, cudaStream_t s) {
     if (grid > ntiles) grid = ntiles;
     if (grid > kMaxBlocksSmallM / 2) grid = kMaxBlocksSmallM / 2;   // the partials hold 2M sums per block
     args.grid_a = (int)grid;
+    args.schedule = DPPF_PATH_TWO_KERNEL;
     general_distance_kernel<M><<<(unsigned)grid, T, 0, s>>>(args);
     general_update_kernel<M><<<(unsigned)grid, T, 0, s>>>(args);
     return cudaGetLastError() == cudaSuccess ? DPPF_OK : DPPF_ERR_CUDA;
@@ -657,6 +666,7 @@ int launch_adamw_round_m(const RoundArgs &a, const AdamArgs &p, int path, int de
     if (grid > kMaxBlocksSmallM) grid = kMaxBlocksSmallM;
     if (path != DPPF_PATH_TWO_KERNEL && coop_supported(dev)) {
         RoundArgs aa = a;
+        aa.schedule = DPPF_PATH_COOPERATIVE;
         AdamArgs pp = p;
         void *params[] = {&aa, &pp};
         if (cudaLaunchCooperativeKernel((const void *)adamw_round_kernel<M>, dim3((unsigned)grid), dim3(T), params, 0,
@@ -664,8 +674,10 @@ int launch_adamw_round_m(const RoundArgs &a, const AdamArgs &p, int path, int de
             return DPPF_OK;
         cudaGetLastError();                              // refused: two plain launches
     }
-    adamw_distance_kernel<M><<<(unsigned)grid, T, 0, s>>>(a, p);
-    adamw_update_kernel<M><<<(unsigned)grid, T, 0, s>>>(a, (int)grid);
+    RoundArgs a2 = a;
+    a2.schedule = DPPF_PATH_TWO_KERNEL;
+    adamw_distance_kernel<M><<<(unsigned)grid, T, 0, s>>>(a2, p);
+    adamw_update_kernel<M><<<(unsigned)grid, T, 0, s>>>(a2, (int)grid);
     return cudaGetLastError() == cudaSuccess ? DPPF_OK : DPPF_ERR_CUDA;
 }
 
@@ -746,6 +758,15 @@ int dppf_consensus_host(float *x_host, int M, int64_t d, int64_t ld, float alpha
     return DPPF_OK;
 }
 
+int dppf_device_schedule(const void *ws, void *cuda_stream) {
+    if (!ws) return DPPF_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    WsHeader h;
+    if (cudaMemcpyAsync(&h, ws, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return -1;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return -1;
+    return h.schedule;
+}
+
 int dppf_device_status(const void *ws, void *cuda_stream) {
     if (!ws) return DPPF_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
@@ -801,6 +822,7 @@ int dppf_distance_partials(const float *x, int M, int64_t d, int64_t ld, double 
     a.norms_stage = reinterpret_cast<float *>(static_cast<unsigned char *>(ws) + norms_stage_offset(M));
     a.M = M;
     a.spin_first = a.spin_later = kSpinLimit;
+    a.schedule = DPPF_PATH_TWO_KERNEL;
     const int grid = launch_distance_only(a, M, dev, s);
     if (grid <= 0) return DPPF_ERR_CUDA;
     const int warps = M < 16 ? M : 16;
@@ -829,6 +851,7 @@ int dppf_update_from_sums(float *x, int M, int64_t d, int64_t ld, float alpha, f
     a.norms_stage = nullptr;
     a.M = M;
     a.spin_first = a.spin_later = kSpinLimit;
+    a.schedule = DPPF_PATH_TWO_KERNEL;
     return launch_update_only(a, M, dev, s);
 }
 

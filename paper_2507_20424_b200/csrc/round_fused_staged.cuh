@@ -101,6 +101,7 @@ __global__ void __launch_bounds__(kStagedThreads, 1) fused_round_kernel_staged(c
             a.hdr->magic = kMagic;
             a.hdr->grid = (int)gridDim.x;
             a.hdr->M = M;
+            a.hdr->schedule = a.schedule;
         }
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // ring B reuses the memory ring A was read from

@@ -41,6 +41,7 @@ struct GeneralArgs {
     WsHeader *hdr;
     double *partials;            // [grid][2 M]: squared distances to x_A, then of the pulled points to P
     int grid_a;                  // two-launch schedule: blocks of the distance launch
+    int schedule;                // DPPF_PATH_* being launched, recorded in the workspace header
 };
 
 // The per-column arithmetic is written once for fp32 and for packed fp32x2: on sm_100 one
@@ -195,6 +196,7 @@ __device__ __forceinline__ void general_write_partials(const GeneralArgs &a, con
         a.hdr->magic = kMagic;
         a.hdr->grid = (int)gridDim.x;
         a.hdr->M = M;
+        a.hdr->schedule = a.schedule;
     }
 }
 

@@ -80,6 +80,7 @@ __global__ void __launch_bounds__(kThreads) distance_kernel_generic(const RoundA
         a.hdr->magic = kMagic;
         a.hdr->grid = (int)gridDim.x;
         a.hdr->M = M;
+        a.hdr->schedule = a.schedule;
     }
 }
 
@@ -155,6 +156,7 @@ __global__ void zero_norms_kernel(float *norms_out, float *norms_stage, WsHeader
         if (norms_out) norms_out[0] = 0.f;
         hdr->status = DPPF_OK;
         hdr->magic = 0;
+        hdr->schedule = DPPF_PATH_TWO_KERNEL;
     }
 }
 

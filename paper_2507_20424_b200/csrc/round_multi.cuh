@@ -38,6 +38,7 @@ struct RoundsArgs {
     WsHeader *hdr;
     double *partials;             // two buffers of [grid, M], the second at partials + partials_half
     long long partials_half;
+    int schedule;                 // DPPF_PATH_* being launched, recorded in the workspace header
     float lambdas[kMaxRoundsPerLaunch];
 };
 
@@ -155,6 +156,7 @@ __global__ void __launch_bounds__(kStagedThreads, 1) rounds_kernel_staged(const 
                 a.hdr->magic = kMagic;
                 a.hdr->grid = (int)gridDim.x;
                 a.hdr->M = M;
+                a.hdr->schedule = a.schedule;
             }
         }
         cg::this_grid().sync();
@@ -276,6 +278,7 @@ __global__ void __launch_bounds__(Tuning<M>::kThreads, Tuning<M>::kBlocksPerSM) 
             a.hdr->magic = kMagic;
             a.hdr->grid = (int)gridDim.x;
             a.hdr->M = M;
+            a.hdr->schedule = a.schedule;
         }
         cg::this_grid().sync();
         for (int m = warp; m < M; m += Tuning<M>::kWarps) {

@@ -156,6 +156,7 @@ __device__ __forceinline__ void distance_pass(const RoundArgs &a, double *s_red 
         a.hdr->magic = kMagic;
         a.hdr->grid = (int)gridDim.x;
         a.hdr->M = M;
+        a.hdr->schedule = a.schedule;
     }
 }
 

@@ -128,6 +128,7 @@ __global__ void __launch_bounds__(kStagedThreads, 1) round_kernel_staged(const R
             a.hdr->magic = kMagic;
             a.hdr->grid = (int)gridDim.x;
             a.hdr->M = M;
+            a.hdr->schedule = a.schedule;
         }
     }
     cg::this_grid().sync();

@@ -85,6 +85,7 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert k(None, 4, 64, 64, 0.1, 0.01, None, X, WS, big, None) == b.ERR_INVALID_ARG
     assert k(V, 4, 64, 64, 0.1, 0.01, None, X + 4, WS, big, None) == b.ERR_ALIGNMENT
     assert lib.dppf_device_status(None, None) == b.ERR_INVALID_ARG
+    assert lib.dppf_device_schedule(None, None) == b.ERR_INVALID_ARG
     gen = lib.dppf_consensus_general
     w_ok = (ctypes.c_float * 4)(1, 2, 3, 4)
     w_zero = (ctypes.c_float * 4)(0, 0, 0, 0)

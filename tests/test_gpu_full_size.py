@@ -19,6 +19,7 @@ def _round_on_gpu(binding, x_np, w, rounds=1):
     for _ in range(rounds):
         binding.dppf_consensus(x, w.alpha, w.lam, norms_out=norms, ws=ws, d=w.d)
     assert binding.dppf_device_status(ws) == binding.OK
+    assert binding.dppf_device_schedule(ws) == binding.PATH_STAGED      # bit-for-bit repeats need the same schedule
     out, r = x.cpu().numpy(), norms.cpu().numpy()
     del x
     torch.cuda.empty_cache()

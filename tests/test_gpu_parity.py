@@ -121,6 +121,23 @@ def test_reproducible_and_schedule_independent(M, d):
     assert np.max(np.abs(e[:, :d].astype(np.float64) - a[:, :d])) <= 1e-8
 
 
+@pytest.mark.parametrize("M,auto", [(4, 3), (8, 3), (16, 3), (20, 1)])
+def test_the_schedule_that_ran_is_recorded(M, auto):
+    """dppf_device_schedule reports what AUTO resolved to and what an explicit request ran."""
+    _, binding = require_gpu()
+    d = 300_001
+    x = to_dev(random_replicas(M, d, seed=3))
+    ws = binding.alloc_workspace(M, d)
+    for path, want in ((0, auto), (1, 1), (2, 2 if M <= 16 else 1), (3, 3 if M <= 16 else 1)):
+        binding.dppf_consensus(x, 0.1, 0.01, ws=ws, d=d, path=path)
+        assert binding.dppf_device_schedule(ws) == want
+    if M <= 16:
+        binding.dppf_consensus_rounds(x, 0.1, 0.01, 3, ws=ws, d=d)
+        assert binding.dppf_device_schedule(ws) == 3
+        binding.dppf_consensus_general(x, 0.1, 0.01, ws=ws, d=d, path=1)
+        assert binding.dppf_device_schedule(ws) == 1
+
+
 def test_norms_out_is_optional_and_iterated_rounds_follow_oracle(oracle):
     import torch
     _, binding = require_gpu()
