@@ -6,7 +6,7 @@
 //   chunk_ring.cuh      shared-memory chunk ring of the staged kernels (bulk async copies, bounded waits)
 //   round_staged.cuh    staged persistent round kernel, one round per launch
 //   round_multi.cuh     several rounds in one launch (update pass of round k + distances of round k+1)
-//   round_fused_staged.cuh  local step (SGD-momentum or AdamW) + round, rows staged through shared memory
+//   round_fused_staged.cuh  SGD-momentum local step + round, x, v, g staged through shared memory
 //   round_general.cuh   general round (weighted consensus variable, push reference, two-term push)
 //   round_generic.cuh   any worker count up to 1024, stand-alone SGD-momentum local step
 //
