@@ -207,6 +207,42 @@ def test_local_steps_then_fused_round(oracle, M, d, tau, path):
     assert same_bits(g_last.cpu().numpy()[:, :d], grads[-1][:, :d])     # gradients are read-only
 
 
+def test_random_shapes_fused_local_step(oracle):
+    """Forty seeded random cases of the fused local step + round over all schedules: worker
+    counts 2..12 (the staged kernel up to 8, the register kernel above), ragged lengths, 1..3 steps."""
+    import torch
+    _, binding = require_gpu()
+    rng = np.random.default_rng(20424_3)
+    for case in range(40):
+        M = int(rng.integers(2, 13))
+        d = int(rng.choice([rng.integers(1, 9), rng.integers(9, 5000), rng.integers(5000, 300_000),
+                            rng.integers(300_000, 2_000_000)]))
+        tau = int(rng.integers(1, 4))
+        path = int(rng.integers(1, 4))
+        w = inputs.WORKLOADS["C3"].scaled(d)
+        w = type(w)(**{**w.__dict__, "M": M})
+        x_np, v_np = inputs.replicas(w, seed=9000 + case), inputs.zeros_like_rows(w)
+        grads = [inputs.gradients(w, t, seed=9000 + case) for t in range(tau)]
+        ref_x, ref_v, r_ref = oracle.local_steps_then_consensus(
+            x_np[:, :d], v_np[:, :d], [g[:, :d] for g in grads], w.lr, w.momentum, w.weight_decay, w.alpha, w.lam)
+        x, v = to_dev(x_np), to_dev(v_np)
+        ws = binding.alloc_workspace(M, d)
+        norms = torch.zeros(M, device="cuda")
+        for t in range(tau - 1):
+            binding.dppf_local_step(x, v, to_dev(grads[t]), w.lr, w.momentum, w.weight_decay, d=d)
+        binding.dppf_local_step_and_consensus(x, v, to_dev(grads[-1]), w.lr, w.momentum, w.weight_decay, w.alpha,
+                                              w.lam, norms_out=norms, ws=ws, d=d, path=path)
+        assert binding.dppf_device_status(ws) == binding.OK
+        info = f"case {case}: M={M} d={d} tau={tau} path={path}"
+        got_x, got_v = x.cpu().numpy(), v.cpu().numpy()
+        assert np.all(np.abs(norms.cpu().numpy() - r_ref) <= 1e-5 * r_ref), info
+        err = np.abs(got_x[:, :d].astype(np.float64) - ref_x[:, :d])
+        assert np.all(err <= 1e-6 * (1 + np.abs(ref_x[:, :d]))), f"{info}: max err {err.max():.3e}"
+        verr = np.abs(got_v[:, :d].astype(np.float64) - ref_v[:, :d])
+        assert np.all(verr <= 1e-6 * (1 + np.abs(ref_v[:, :d]))), info
+        assert_pad_untouched(got_x, d), assert_pad_untouched(got_v, d)
+
+
 def test_fused_matches_unfused_sequence():
     """Local step then round as two calls vs the fused call: the momentum buffers agree bit
     for bit (same arithmetic); the replicas agree to rounding of the distances (the two

@@ -132,3 +132,53 @@ def test_norms_out_is_optional_and_bad_arguments_are_refused():
         binding.dppf_consensus_rounds(x, float("nan"), 0.01, 2, d=d)
     torch.cuda.synchronize()
     assert same_bits(x.cpu().numpy()[:, :d], a[:, :d])
+
+
+def test_random_shapes_rounds_and_schedules(oracle):
+    """Sixty seeded random cases: worker counts 2..16, vector lengths that straddle the tail
+    columns, one chunk, one ring and several rings per block, 1..6 rounds, every schedule."""
+    _, binding = require_gpu()
+    rng = np.random.default_rng(20424_7)
+    for case in range(60):
+        M = int(rng.integers(2, 17))
+        d = int(rng.choice([rng.integers(1, 9), rng.integers(9, 5000), rng.integers(5000, 400_000),
+                            rng.integers(400_000, 3_000_000)]))
+        n = int(rng.integers(1, 7))
+        alpha = float(rng.choice([0.05, 0.1, 0.5, 0.9]))
+        lam = float(rng.choice([0.0, 0.01, 0.05, 0.5]))
+        if lam == 0.0:
+            alpha = min(alpha, 0.1)     # a strong pull with no push collapses the replicas to within a few
+                                        # fp32 ulps of each other, where no distance has five good digits
+        path = int(rng.integers(1, 4))
+        x = replicas(M, d, seed=5000 + case)
+        ref, rs = oracle_rounds(oracle, x, alpha, [lam] * n, d)
+        got, norms = gpu_rounds(binding, x, d, alpha, lam, n, path)
+        info = f"case {case}: M={M} d={d} n={n} alpha={alpha} lam={lam} path={path}"
+        assert np.all(np.abs(norms - rs) <= 1e-5 * rs), info
+        err = np.abs(got[:, :d].astype(np.float64) - ref[:, :d])
+        assert np.all(err <= 1e-6 * (1 + np.abs(ref[:, :d]))), f"{info}: max err {err.max():.3e}"
+        assert_pad_untouched(got, d)
+
+
+def test_rounds_call_replayed_from_a_cuda_graph():
+    """Once the first call on the device has been made, a multi-round call can be stream-captured;
+    the replay gives the eager result bit for bit."""
+    import torch
+    _, binding = require_gpu()
+    d = 1_000_003
+    x_np = replicas(4, d, seed=37)
+    ws = binding.alloc_workspace(4, d)
+    norms = torch.zeros(6, 4, device="cuda")
+    eager = to_dev(x_np)
+    binding.dppf_consensus_rounds(eager, 0.1, 0.005, 6, norms_out=norms, ws=ws, d=d)
+    eager_norms = norms.clone()
+    x = to_dev(x_np)
+    static = x.clone()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        binding.dppf_consensus_rounds(static, 0.1, 0.005, 6, norms_out=norms, ws=ws, d=d)
+    static.copy_(x)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert same_bits(static.cpu().numpy()[:, :d], eager.cpu().numpy()[:, :d])
+    assert torch.equal(norms, eager_norms)
