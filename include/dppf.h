@@ -96,7 +96,8 @@ int dppf_consensus(float *x, int M, int64_t d, int64_t ld, float alpha, float la
  * run to run; TWO_KERNEL and COOPERATIVE agree bit for bit, STAGED groups the sums of
  * squares differently and may differ from them in the last bits of r_m.  If the runtime
  * refuses a cooperative launch (its blocks cannot all be resident, e.g. SMs shared with
- * another client) the call falls back to the two-launch schedule. */
+ * another client) the call falls back to the two-launch schedule; dppf_device_schedule
+ * tells which schedule ran. */
 int dppf_consensus_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,
                       float *norms_out, void *ws, size_t ws_bytes, int path, void *cuda_stream);
 

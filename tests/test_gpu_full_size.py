@@ -51,23 +51,36 @@ def test_c5_identical_replicas_round_is_bit_exact(oracle):
     assert_pad_untouched(got, w.d)
 
 
-def test_c4_first_and_hundredth_round(oracle):
-    """100 rounds back to back on the device; the oracle iterates 100 times too."""
-    _, binding = require_gpu()
+@pytest.fixture(scope="module")
+def c4_oracle_rounds(oracle):
+    """The oracle's round applied 100 times to the ViT-B/16-sized workload (about 45 s of CPU
+    work, shared by the tests below): the input, the state after round 1, the final state and
+    the distances before every round."""
     w = inputs.WORKLOADS["C4"]
     x = inputs.replicas(w)
-    ref, r_ref, _ = oracle.consensus_blocked(x, w.alpha, w.lam, d=w.d)
-    got, r = _round_on_gpu(binding, x, w, rounds=1)
-    assert_parity(got, r, ref, r_ref, w.d)
-    np.testing.assert_allclose(r, w.drift_std * np.sqrt(w.d * (w.M - 1) / w.M), rtol=0.01)   # 8.058
-    for _ in range(w.rounds - 1):
+    ref, first, rs = x, None, []
+    for k in range(w.rounds):
         ref, r_ref, _ = oracle.consensus_blocked(ref, w.alpha, w.lam, d=w.d)
+        rs.append(r_ref)
+        if k == 0:
+            first = ref
+    return x, first, ref, np.array(rs)
+
+
+def test_c4_first_and_hundredth_round(c4_oracle_rounds):
+    """100 rounds back to back on the device, one call per round; the oracle iterates 100 times too."""
+    _, binding = require_gpu()
+    w = inputs.WORKLOADS["C4"]
+    x, first, last, rs = c4_oracle_rounds
+    got, r = _round_on_gpu(binding, x, w, rounds=1)
+    assert_parity(got, r, first, rs[0], w.d)
+    np.testing.assert_allclose(r, w.drift_std * np.sqrt(w.d * (w.M - 1) / w.M), rtol=0.01)   # 8.058
     got, r = _round_on_gpu(binding, x, w, rounds=w.rounds)
-    assert_parity(got, r, ref, r_ref, w.d)      # r holds the distances before round 100
+    assert_parity(got, r, last, rs[-1], w.d)      # r holds the distances before round 100
     assert_pad_untouched(got, w.d)
     # the valley width has contracted toward lambda/alpha (Theorem 1): r_100 - 0.05 = 0.9^99 (r_1 - 0.05)
     a, l = float(np.float32(w.alpha)), float(np.float32(w.lam))
-    assert np.all(np.abs(r_ref - l / a) < 1e-3)
+    assert np.all(np.abs(rs[-1] - l / a) < 1e-3)
 
 
 def test_c3_eight_local_steps_then_fused_round(oracle):
@@ -146,19 +159,14 @@ def test_rows_longer_than_2_to_31_columns(oracle, path):
 
 # ---------------------------------------------------------------- several rounds per launch
 
-def test_c4_hundred_rounds_in_one_call(oracle):
+def test_c4_hundred_rounds_in_one_call(c4_oracle_rounds):
     """The 100 back-to-back rounds of the ViT-B/16-sized workload as ONE dppf_consensus_rounds call
     (what the benchmark's multi_round figure times): the replicas after round 100 and the
     distances before every one of the 100 rounds against the oracle iterated 100 times."""
     import torch
     _, binding = require_gpu()
     w = inputs.WORKLOADS["C4"]
-    x_np = inputs.replicas(w)
-    ref, rs = x_np, []
-    for _ in range(w.rounds):
-        ref, r_ref, _ = oracle.consensus_blocked(ref, w.alpha, w.lam, d=w.d)
-        rs.append(r_ref)
-    rs = np.array(rs)
+    x_np, _, ref, rs = c4_oracle_rounds
     outs = []
     for _ in range(2):
         x = to_dev(x_np)

@@ -208,15 +208,15 @@ def test_local_steps_then_fused_round(oracle, M, d, tau, path):
 
 
 def test_random_shapes_fused_local_step(oracle):
-    """Forty seeded random cases of the fused local step + round over all schedules: worker
+    """Thirty seeded random cases of the fused local step + round over all schedules: worker
     counts 2..12 (the staged kernel up to 8, the register kernel above), ragged lengths, 1..3 steps."""
     import torch
     _, binding = require_gpu()
     rng = np.random.default_rng(20424_3)
-    for case in range(40):
+    for case in range(30):
         M = int(rng.integers(2, 13))
         d = int(rng.choice([rng.integers(1, 9), rng.integers(9, 5000), rng.integers(5000, 300_000),
-                            rng.integers(300_000, 2_000_000)]))
+                            rng.integers(300_000, 1_200_000)]))
         tau = int(rng.integers(1, 4))
         path = int(rng.integers(1, 4))
         w = inputs.WORKLOADS["C3"].scaled(d)
