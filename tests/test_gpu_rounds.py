@@ -182,3 +182,34 @@ def test_rounds_call_replayed_from_a_cuda_graph():
     torch.cuda.synchronize()
     assert same_bits(static.cpu().numpy()[:, :d], eager.cpu().numpy()[:, :d])
     assert torch.equal(norms, eager_norms)
+
+
+@pytest.mark.parametrize("M,path", [(4, 3), (8, 3), (3, 2), (16, 3)])
+def test_distances_follow_the_closed_form_of_theorem_1(M, path):
+    """No oracle involved: on a centred regular simplex the unit directions sum to zero, so the
+    average never moves and every distance obeys r_k = lambda/alpha + (1-alpha)^k (r_0 - lambda/alpha)
+    (proof of Theorem 1); with lambda = 0.5, alpha = 0.1 it settles at the 5 the paper prints."""
+    import torch
+    _, binding = require_gpu()
+    d, n, alpha, lam, r0 = 120_000 // M * M, 60, 0.1, 0.5, 2.0
+    block = d // M
+    e = np.zeros((M, d))
+    for m in range(M):
+        e[m, m * block:(m + 1) * block] = 1.0 / np.sqrt(block)        # orthonormal rows
+    centred = e - e.mean(axis=0)
+    centred *= r0 / np.linalg.norm(centred[0])
+    x_np = padded((0.3 + centred).astype(np.float32))
+    x = to_dev(x_np)
+    norms = torch.zeros(n, M, device="cuda")
+    ws = binding.alloc_workspace(M, d)
+    binding.dppf_consensus_rounds(x, alpha, lam, n, norms_out=norms, ws=ws, d=d, path=path)
+    assert binding.dppf_device_status(ws) == binding.OK
+    r = norms.cpu().numpy().astype(np.float64)
+    a32, l32 = float(np.float32(alpha)), float(np.float32(lam))
+    r_start = np.linalg.norm(x_np[:, :d].astype(np.float64) - x_np[:, :d].astype(np.float64).mean(axis=0), axis=1)
+    k = np.arange(n)[:, None]
+    want = l32 / a32 + (1.0 - a32) ** k * (r_start[None, :] - l32 / a32)
+    np.testing.assert_allclose(r, want, rtol=2e-5)
+    assert abs(want[-1, 0] - 5.0) < 0.01                               # 5 = lambda / alpha
+    mean_after = x.cpu().numpy()[:, :d].astype(np.float64).mean(axis=0)
+    np.testing.assert_allclose(mean_after, x_np[:, :d].astype(np.float64).mean(axis=0), atol=2e-6)
