@@ -275,6 +275,23 @@ def time_oracle(w, variant, seed, budget_s):
     return 1.0 / (dt * w.d / d_s), cores, d_s, dt * reps
 
 
+def single_thread_oracle_rate(w, seed, budget_s):
+    """Full-workload rounds/s of the oracle's round on ONE thread, from a column slice."""
+    import numpy as np
+    import oracle
+    from paper_2507_20424_b200 import inputs
+    probe = min(w.d, 500_000)
+    x = np.ascontiguousarray(inputs.replicas(w.scaled(probe), seed)[:, :probe])
+    t0 = time.perf_counter()
+    oracle.consensus_blocked(x, w.alpha, w.lam, d=probe, threads=1)
+    rate = probe / max(time.perf_counter() - t0, 1e-6)
+    d_s = int(min(w.d, max(probe, rate * budget_s)))
+    x = np.ascontiguousarray(inputs.replicas(w.scaled(d_s), seed)[:, :d_s])
+    t0 = time.perf_counter()
+    oracle.consensus_blocked(x, w.alpha, w.lam, d=d_s, threads=1)
+    return 1.0 / ((time.perf_counter() - t0) * w.d / d_s)
+
+
 def run_reference(args):
     """The CPU oracle as the reference arm: rank 0 only, bounded column slice per step."""
     rank = int(os.environ.get("RANK", "0"))
@@ -365,6 +382,8 @@ def run_ours(args):
         val, cores, d_s, dt = time_oracle(w, variant, seed, budget_s=12.0)
         cpu = {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"oracle steps on the first {d_s} of {w.d} columns for {dt:.1f} s, rate scaled by columns"}
+        if variant == "plain" and w.tau == 0:      # the same oracle on one thread, on a shorter slice
+            cpu["single_thread_value"] = single_thread_oracle_rate(w, seed, budget_s=5.0)
 
     torch.cuda.set_device(local)
     if world > 1:
