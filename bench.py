@@ -89,11 +89,11 @@ def measured_peaks():
 NCU_TRAFFIC = {
     ("C4", 86_567_656, "round_kernel_staged"): 4.008e9,
     ("C4", 86_567_656, "rounds100"): 264.5e9,
-    ("C2", 26_200_000, "round_kernel_staged"): 2.368e9,
+    ("C2", 26_200_000, "round_kernel_staged"): 2.369e9,
     ("C5", 44_549_160, "rounds_kernel_staged"): 8.411e9,
     ("C3", 25_557_032, "fused_round_kernel_staged"): 2.746e9,
-    ("C4", 86_567_656, "general_round_kernel"): 4.007e9,
-    ("C4", 86_567_656, "adamw_round_kernel"): 12.364e9,
+    ("C4", 86_567_656, "general_round_kernel"): 4.004e9,
+    ("C4", 86_567_656, "adamw_round_kernel"): 12.365e9,
 }
 
 
