@@ -138,6 +138,37 @@ def test_the_schedule_that_ran_is_recorded(M, auto):
         assert binding.dppf_device_schedule(ws) == 1
 
 
+@pytest.mark.parametrize("path", PATHS)
+def test_resuming_from_a_saved_state_reproduces_the_run_bit_for_bit(path):
+    """Checkpoint / resume: the state of the path is x (and v with the fused step); ten rounds in
+    a row equal five rounds, a copy of the replicas through host memory into fresh buffers and a
+    fresh workspace, and five more rounds."""
+    import torch
+    _, binding = require_gpu()
+    d = 700_001
+    w = inputs.WORKLOADS["C3"].scaled(d)
+    x_np, v_np = random_replicas(4, d, seed=21), inputs.zeros_like_rows(w)
+    g = to_dev(inputs.gradients(w, 0))
+
+    def rounds(x, v, ws, k):
+        for _ in range(k):
+            binding.dppf_consensus(x, 0.1, 0.005, ws=ws, d=d, path=PATHS[path])
+            binding.dppf_local_step_and_consensus(x, v, g, w.lr, w.momentum, w.weight_decay, 0.1, 0.005, ws=ws,
+                                                  d=d, path=PATHS[path])
+
+    xa, va = to_dev(x_np), to_dev(v_np)
+    rounds(xa, va, binding.alloc_workspace(4, d), 10)
+    xb, vb = to_dev(x_np), to_dev(v_np)
+    rounds(xb, vb, binding.alloc_workspace(4, d), 5)
+    saved_x, saved_v = xb.cpu().numpy().copy(), vb.cpu().numpy().copy()
+    del xb, vb
+    torch.cuda.empty_cache()
+    xc, vc = to_dev(saved_x), to_dev(saved_v)
+    rounds(xc, vc, binding.alloc_workspace(4, d), 5)
+    assert same_bits(xa.cpu().numpy()[:, :d], xc.cpu().numpy()[:, :d])
+    assert same_bits(va.cpu().numpy()[:, :d], vc.cpu().numpy()[:, :d])
+
+
 def test_norms_out_is_optional_and_iterated_rounds_follow_oracle(oracle):
     import torch
     _, binding = require_gpu()
