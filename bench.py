@@ -25,7 +25,10 @@ Multi-GPU: by default the path does not shard (one GPU holds all M replicas of a
 N > 1 runs N independent replicas, one process per GPU, with no data-path collective ("weak"
 scaling: rounds/s adds up).  --shard columns splits the columns of ONE workload over the N
 ranks instead: every step is dppf_distance_partials, an all-reduce of the M fp64 sums of
-squares, dppf_update_from_sums ("strong" scaling).
+squares, dppf_update_from_sums ("strong" scaling).  --shard workers is the paper's own
+arrangement, one replica per GPU (needs N = M ranks): every step is an all-reduce (sum) of the
+d parameters and dppf_worker_update; with N = 1 the all-reduce is left out and only the
+worker kernel is timed.
 
 ``--impl reference`` times the CPU oracle (plain C, fp64) on the host cores on a
 bounded column slice of the same workload; rank 0 only.
@@ -58,7 +61,7 @@ def parse_args(argv=None):
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
     p.add_argument("--workload", default="C4")
     p.add_argument("--variant", default="plain", choices=["plain", "general", "adamw"])
-    p.add_argument("--shard", default="none", choices=["none", "columns"])
+    p.add_argument("--shard", default="none", choices=["none", "columns", "workers"])
     p.add_argument("--d", type=int, default=0, help="override the vector length (profiling on a smaller case)")
     p.add_argument("--path", default="auto", choices=["auto", "two_kernel", "cooperative", "staged"])
     p.add_argument("--rounds-per-call", type=int, default=100, help="rounds per dppf_consensus_rounds call")
@@ -367,11 +370,14 @@ def run_ours(args):
     binding.load(rebuild_if_stale=True)
     w = workload_of(args)
     sharded = args.shard == "columns"
+    per_worker = args.shard == "workers"
     variant = args.variant
-    if sharded and (variant != "plain" or w.tau > 0):
-        raise SystemExit("--shard columns applies to the plain round")
+    if (sharded or per_worker) and (variant != "plain" or w.tau > 0):
+        raise SystemExit("--shard applies to the plain round")
+    if per_worker and world not in (1, w.M):
+        raise SystemExit(f"--shard workers needs one rank per worker ({w.M}) or a single rank")
     # replicas-only runs give every rank its own replica set; column shards share one
-    seed = (inputs.DEFAULT_SEED if args.seed is None else args.seed) + (0 if sharded else rank)
+    seed = (inputs.DEFAULT_SEED if args.seed is None else args.seed) + (0 if (sharded or per_worker) else rank)
     path = {"auto": binding.PATH_AUTO, "two_kernel": binding.PATH_TWO_KERNEL,
             "cooperative": binding.PATH_COOPERATIVE, "staged": binding.PATH_STAGED}[args.path]
 
@@ -400,7 +406,27 @@ def run_ours(args):
     fused_sgd = variant == "plain" and w.tau > 0
     staged = args.path in ("auto", "staged") and w.M <= 16
 
-    if sharded:
+    if per_worker:
+        # this rank's replica as a flat vector; the reduced vector is what a sum all-reduce leaves
+        xw = torch.from_numpy(np.ascontiguousarray(x_host[rank, :w.d])).cuda()
+        red = torch.from_numpy(np.ascontiguousarray(x_host[:, :w.d].astype(np.float64).sum(axis=0)
+                                                    .astype(np.float32))).cuda()
+        ws = binding.alloc_workspace(1, w.d)
+        norms = torch.zeros(1, device="cuda")
+        B = w.d * 4
+        model_units, kernel_id = 5.0, "worker_round_kernel"
+        kernel_name = ("all-reduce (sum) of the d parameters, then worker_round_kernel (distance pass, grid barrier, "
+                       "update pass on this worker's replica)" if world > 1 else
+                       "worker_round_kernel (distance pass, grid barrier, update pass on one replica; the all-reduce "
+                       "is left out on a single GPU)")
+        launches_per_step = 1
+
+        def step():
+            if world > 1:
+                red.copy_(xw)
+                dist.all_reduce(red)
+            binding.dppf_worker_update(xw, red, 1.0 / w.M, w.alpha, w.lam, norm_out=norms, ws=ws)
+    elif sharded:
         sums = torch.zeros(w.M, dtype=torch.float64, device="cuda")
         model_units, kernel_id = 3.0, "distance_kernel + update_kernel (column shard)"
         kernel_name = ("dppf_distance_partials (distance_kernel + sum_partials_kernel), all-reduce of M fp64 sums, "
@@ -495,7 +521,7 @@ def run_ours(args):
     # the same rounds, rounds_per_call of them per library call (update pass of round k fused with
     # the distance pass of round k + 1): (1 + 2n) x M d 4 bytes per call
     multi_round = None
-    if variant == "plain" and not fused_sgd and not sharded and not args.no_multi_round and w.M <= 16:
+    if variant == "plain" and not fused_sgd and not sharded and not per_worker and not args.no_multi_round and w.M <= 16:
         n = args.rounds_per_call
         norms_all = torch.zeros(n, w.M, device="cuda")
         binding.dppf_consensus_rounds(x, w.alpha, w.lam, n, norms_out=norms_all, ws=ws, d=w.d)
@@ -524,7 +550,7 @@ def run_ours(args):
 
     # optional: the same K steps captured once into a CUDA graph and replayed (launch overhead off the host)
     graph_replay = None
-    if args.graph and not sharded and variant != "adamw":
+    if args.graph and not sharded and not per_worker and variant != "adamw":
         chunk = min(K, 100)
         cg_ = torch.cuda.CUDAGraph()
         with torch.cuda.graph(cg_):
@@ -546,7 +572,7 @@ def run_ours(args):
     # end-to-end: replicas live in pinned host memory; every step copies them in, runs the
     # round and copies the replicas and the M distances back.
     e2e = None
-    if not args.no_e2e and variant == "plain" and not fused_sgd and not sharded:
+    if not args.no_e2e and variant == "plain" and not fused_sgd and not sharded and not per_worker:
         norms_host = torch.zeros(w.M).pin_memory()
         binding.dppf_consensus_host(x_pinned, w.alpha, w.lam, norms_host, x, ws, d=w.d)
         fence()
@@ -561,16 +587,18 @@ def run_ours(args):
                "h2d_bytes_per_step": B, "d2h_bytes_per_step": B + 4 * w.M, "steps": args.e2e_steps}
 
     if rank == 0:
-        jobs = 1 if sharded else world                   # column shards: all ranks work on ONE round
+        jobs = 1 if (sharded or per_worker) else world   # shards: all ranks work on ONE round
         achieved = model_units * B / (per_launch_ms * 1e-3) / 1e9
         value = whole_job_rate(K, jobs, total_ms)
         model_gbs = model_units * B * K / (total_ms * 1e-3) / 1e9
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
                 "warmup": max(3, args.warmup), "repeats": R, "ms_per_step": total_ms / K,
                 "ms_per_step_min_max": [min(rep_ms) / K, max(rep_ms) / K],
-                "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
+                "higher_is_better": True, "scaling": "strong" if (sharded or per_worker) else "weak", "vs_baseline": None,
                 "dtype": "f32", "data": "synthetic", "config": config_of(w, variant),
-                "parallelism": (f"column shards x{world} (all-reduce of {w.M} fp64 sums per round)" if sharded else
+                "parallelism": (f"one replica per GPU x{world} (all-reduce of d fp32 per round)" if per_worker and world > 1
+                                else "one replica of the workload on one GPU (no all-reduce)" if per_worker else
+                                f"column shards x{world} (all-reduce of {w.M} fp64 sums per round)" if sharded else
                                 f"replicas x{world}" if world > 1 else "single GPU"),
                 "schedule": args.path,
                 "model_gbs_per_gpu": model_gbs, "frac_of_nominal_8tbs": model_gbs / NOMINAL_HBM_GBS,

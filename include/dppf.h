@@ -102,6 +102,23 @@ int dppf_consensus_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float
                       float *norms_out, void *ws, size_t ws_bytes, int path, void *cuda_stream);
 
 /*
+ * One worker's share of a round when every GPU holds ONE replica, the arrangement the paper
+ * itself runs (Algorithm 1: the workers obtain the consensus variable with one collective per
+ * round, then each pulls and pushes its own replica; Sec. 5 single-line update):
+ *   x          device fp32[d], 128-byte aligned: this worker's replica, updated in place
+ *   x_reduced  device fp32[d], 128-byte aligned: the all-reduced parameters of all workers;
+ *              x_A = scale * x_reduced (scale = 1/M after a sum all-reduce, 1 after a mean)
+ *   norm_out   NULL, or device fp32[1]: r = ||x - x_A|| before the update
+ *   r <- ||x - x_A||,  x <- x + (x_A - x)(alpha - lambda / r);  r == 0 leaves x untouched.
+ * The collective is the caller's (e.g. an NCCL all-reduce of the d floats on the same stream,
+ * issued before this call); no second exchange is needed, because each worker's norm only
+ * involves its own replica and x_A.  One cooperative launch (two launches if refused),
+ * 5 d 4 bytes of traffic.  ws: dppf_workspace_bytes(1, d).  x, x_reduced, ws must not overlap.
+ */
+int dppf_worker_update(float *x, const float *x_reduced, float scale, int64_t d, float alpha,
+                       float lambda, float *norm_out, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * n_rounds pull-push rounds back to back on x[M, ld], as ONE device pass sequence: the
  * single-line update of Sec. 5 applied n_rounds times, every round from its own pre-round
  * average (proof of Theorem 1, first display; the noise-free iteration whose distances the

@@ -15,6 +15,8 @@ Every function follows one passage of the paper:
   the optimiser stated in ``dppf_oracle.c``) followed by the round.
 * ``consensus_blocked``    -- the same round with the sum over coordinates
   grouped into per-thread column blocks (OpenMP), for timing and large cases.
+* ``worker_update``        -- the single-line update (Sec. 5) of ONE worker given the
+  average, as each worker applies it in Algorithm 1 after the collective (numpy, fp64).
 """
 from __future__ import annotations
 
@@ -198,3 +200,20 @@ def local_steps_then_consensus(x, v, grads, lr, momentum, weight_decay, alpha, l
     x64, v64 = local_steps_f64(x, v, grads, lr, momentum, weight_decay, d)
     out, r = consensus_f64(x64, alpha, lam, d)
     return out, v64, r
+
+
+def worker_update(x, reduced, scale, alpha, lam):
+    """One worker's pull-push update given the all-reduced parameters (Algorithm 1 after
+    "obtain x_C" with x_C = x_A; Sec. 5 single-line update): x_A = scale * reduced,
+    r = ||x - x_A||, x_plus = x + (x_A - x)(alpha - lam / r); r == 0 leaves x as it is.
+    ``x`` and ``reduced`` are fp32 vectors, the scalars are rounded to fp32 first (they cross
+    the C ABI as floats) and everything else is fp64.  Returns (x_plus fp32, r fp64)."""
+    x32 = np.asarray(x, dtype=np.float32)
+    a_vec = np.float64(np.float32(scale)) * np.asarray(reduced, dtype=np.float32).astype(np.float64)
+    x64 = x32.astype(np.float64)
+    gap = a_vec - x64
+    r = float(np.sqrt(np.sum(gap * gap)))
+    if not r > 0.0:
+        return x32.copy(), 0.0
+    c = np.float64(np.float32(alpha)) - np.float64(np.float32(lam)) / r
+    return (x64 + gap * c).astype(np.float32), r

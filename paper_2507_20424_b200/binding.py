@@ -21,7 +21,7 @@ EXPORTS = ("dppf_workspace_bytes", "dppf_consensus", "dppf_consensus_ex", "dppf_
            "dppf_local_step_and_consensus", "dppf_local_step_and_consensus_ex",
            "dppf_consensus_host", "dppf_device_status", "dppf_device_schedule", "dppf_status_string", "dppf_launch_count",
            "dppf_consensus_static", "dppf_static_device_status", "dppf_consensus_general", "dppf_consensus_general_ex",
-           "dppf_distance_partials", "dppf_update_from_sums", "dppf_adamw_step_and_consensus_ex",
+           "dppf_distance_partials", "dppf_update_from_sums", "dppf_worker_update", "dppf_adamw_step_and_consensus_ex",
            "dppf_consensus_rounds", "dppf_consensus_rounds_ex", "dppf_debug_set_poll_limits",
            "dppf_adamw_step", "dppf_adamw_step_and_consensus",
            "dppf_lambda_schedule", "dppf_lr_cosine", "dppf_qsr_period", "dppf_round_metrics")
@@ -88,6 +88,8 @@ def load(rebuild_if_stale: bool = False) -> ctypes.CDLL:
     lib.dppf_distance_partials.restype = i32
     lib.dppf_update_from_sums.argtypes = [vp, i32, i64, i64, f32, f32, vp, vp, vp]
     lib.dppf_update_from_sums.restype = i32
+    lib.dppf_worker_update.argtypes = [vp, vp, f32, i64, f32, f32, vp, vp, sz, vp]
+    lib.dppf_worker_update.restype = i32
     lib.dppf_static_device_status.argtypes = [vp]
     lib.dppf_static_device_status.restype = i32
     lib.dppf_consensus_general_ex.argtypes = [vp, i32, i64, i64, f32, f32, ctypes.POINTER(f32), i32, i32, vp, vp,
@@ -202,6 +204,21 @@ def dppf_update_from_sums(x, alpha, lam, sums, norms_out=None, d=None):
         raise ValueError("sums must be an fp64 CUDA tensor with M entries")
     _check(load().dppf_update_from_sums(x.data_ptr(), M, d, ld, alpha, lam, sums.data_ptr(), _ptr(norms_out),
                                         _stream()), "dppf_update_from_sums")
+
+
+def dppf_worker_update(x, x_reduced, scale, alpha, lam, norm_out=None, ws=None):
+    """This worker's pull-push update from the all-reduced parameters (one replica per GPU):
+    ``x`` and ``x_reduced`` are 1-D fp32 CUDA tensors of the same length; x_A = scale * x_reduced."""
+    for t in (x, x_reduced):
+        if t.dim() != 1 or t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
+            raise ValueError("expected contiguous 1-D fp32 CUDA tensors")
+    if x.numel() != x_reduced.numel():
+        raise ValueError("x and x_reduced must have the same length")
+    d = x.numel()
+    ws = alloc_workspace(1, d, x.device) if ws is None else ws
+    _check(load().dppf_worker_update(x.data_ptr(), x_reduced.data_ptr(), scale, d, alpha, lam, _ptr(norm_out),
+                                     ws.data_ptr(), ws.numel(), _stream()), "dppf_worker_update")
+    return ws
 
 
 def debug_set_poll_limits(first_pass_polls=-1, later_pass_polls=-1) -> None:

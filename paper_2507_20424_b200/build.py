@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 SOURCES = [os.path.join(_PKG, "csrc", "dppf.cu")]          # one translation unit ...
 HEADERS = [os.path.join(_ROOT, "include", "dppf.h")] + [    # ... that includes the kernel families
     os.path.join(_PKG, "csrc", n) for n in ("common.cuh", "round_register.cuh", "adamw.cuh", "chunk_ring.cuh", "round_staged.cuh",
-                                            "round_multi.cuh", "round_fused_staged.cuh", "round_general.cuh", "round_generic.cuh")]
+                                            "round_multi.cuh", "round_fused_staged.cuh", "round_general.cuh", "round_generic.cuh", "round_worker.cuh")]
 LIB_PATH = os.path.join(_PKG, "libdppf.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -9,6 +9,7 @@
 //   round_fused_staged.cuh  SGD-momentum local step + round, x, v, g staged through shared memory
 //   round_general.cuh   general round (weighted consensus variable, push reference, two-term push)
 //   round_generic.cuh   any worker count up to 1024, stand-alone SGD-momentum local step
+//   round_worker.cuh    one worker's update from the all-reduced parameters (one replica per GPU)
 //
 // Data layout: x[M, ld] fp32, one row per worker, rows 128-byte aligned.  A "vector" is
 // one float4 (four consecutive columns of one row); a thread always handles the same
@@ -41,6 +42,7 @@
 #include "round_fused_staged.cuh"
 #include "round_general.cuh"
 #include "round_generic.cuh"
+#include "round_worker.cuh"
 
 namespace {
 
@@ -642,6 +644,7 @@ int launch_adamw_step(float *x, const AdamArgs &p, int M, int64_t d, int64_t ld,
 }
 
 std::atomic<int> g_adamw_occ[64][kMaxTemplateM + 1];
+std::atomic<int> g_worker_occ[64];
 
 template <int M>
 int launch_adamw_round_m(const RoundArgs &a, const AdamArgs &p, int path, int dev, cudaStream_t s) {
@@ -853,6 +856,67 @@ int dppf_update_from_sums(float *x, int M, int64_t d, int64_t ld, float alpha, f
     a.spin_first = a.spin_later = kSpinLimit;
     a.schedule = DPPF_PATH_TWO_KERNEL;
     return launch_update_only(a, M, dev, s);
+}
+
+// ---- one replica per GPU: this worker's pull-push update from the all-reduced parameters
+
+int dppf_worker_update(float *x, const float *x_reduced, float scale, int64_t d, float alpha, float lambda,
+                       float *norm_out, void *ws, size_t ws_bytes, void *cuda_stream) {
+    int rc = check_layout(x, 1, d, (d + 31) / 32 * 32);
+    if (rc != DPPF_OK) return rc;
+    if (!x_reduced) return DPPF_ERR_INVALID_ARG;
+    if (!aligned128(x_reduced)) return DPPF_ERR_ALIGNMENT;
+    if (!finite_all({scale, alpha, lambda})) return DPPF_ERR_INVALID_ARG;
+    if (!ws) return DPPF_ERR_INVALID_ARG;
+    if (!aligned128(ws)) return DPPF_ERR_ALIGNMENT;
+    if (ws_bytes < workspace_bytes(1)) return DPPF_ERR_WORKSPACE;
+    const size_t bytes = (size_t)d * sizeof(float);
+    if (overlap(x, bytes, x_reduced, bytes) || overlap(x, bytes, ws, workspace_bytes(1)) ||
+        overlap(x_reduced, bytes, ws, workspace_bytes(1)))
+        return DPPF_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DPPF_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const int sms = sm_count(dev);
+    if (sms <= 0) return DPPF_ERR_CUDA;
+    RoundArgs a;
+    a.x = x; a.v = nullptr; a.g = x_reduced;
+    a.d = d; a.ld = d; a.nvec = d / 4;
+    a.alpha = alpha; a.lambda = lambda; a.lr = scale; a.mu = a.wd = 0.f;
+    a.norms_out = norm_out;
+    a.hdr = reinterpret_cast<WsHeader *>(ws);
+    a.partials = reinterpret_cast<double *>(static_cast<unsigned char *>(ws) + kHeaderBytes);
+    a.norms_stage = reinterpret_cast<float *>(static_cast<unsigned char *>(ws) + norms_stage_offset(1));
+    a.M = 1;
+    a.spin_first = a.spin_later = kSpinLimit;
+    const long long tile_vecs = (long long)kWorkerThreads * kWorkerUnroll;
+    long long ntiles = (a.nvec + tile_vecs - 1) / tile_vecs;
+    if (ntiles < 1) ntiles = 1;
+    int per_sm = g_worker_occ[dev].load(std::memory_order_relaxed);
+    if (per_sm == 0) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, worker_round_kernel, kWorkerThreads, 0) !=
+                cudaSuccess || per_sm < 1) {
+            cudaGetLastError();
+            return DPPF_ERR_CUDA;
+        }
+        g_worker_occ[dev].store(per_sm, std::memory_order_relaxed);
+    }
+    if (per_sm > kWorkerBlocksPerSM) per_sm = kWorkerBlocksPerSM;
+    long long grid = (long long)sms * per_sm;
+    if (grid > ntiles) grid = ntiles;
+    if (grid > kMaxBlocksSmallM) grid = kMaxBlocksSmallM;
+    if (coop_supported(dev)) {
+        a.schedule = DPPF_PATH_COOPERATIVE;
+        void *params[] = {&a};
+        if (cudaLaunchCooperativeKernel((const void *)worker_round_kernel, dim3((unsigned)grid), dim3(kWorkerThreads),
+                                        params, 0, s) == cudaSuccess)
+            return DPPF_OK;
+        cudaGetLastError();
+    }
+    a.schedule = DPPF_PATH_TWO_KERNEL;
+    worker_distance_kernel<<<(unsigned)grid, kWorkerThreads, 0, s>>>(a);
+    worker_update_kernel<<<(unsigned)grid, kWorkerThreads, 0, s>>>(a, (int)grid);
+    return cudaGetLastError() == cudaSuccess ? DPPF_OK : DPPF_ERR_CUDA;
 }
 
 int dppf_consensus_rounds_ex(float *x, int M, int64_t d, int64_t ld, float alpha, float lambda,

@@ -123,3 +123,42 @@ def test_column_shard_covers_every_column_once():
             for (lo, hi), (lo2, _) in zip(spans[:-1], spans[1:]):
                 assert hi == lo2 and lo <= hi
             assert all(lo % 32 == 0 or lo == hi for lo, hi in spans)      # non-empty shards start on 128 bytes
+
+
+WORKER_PER_RANK = r"""
+import os, sys, json
+sys.path.insert(0, sys.argv[1])
+import numpy as np
+import torch, torch.distributed as dist
+import oracle
+from paper_2507_20424_b200 import inputs
+rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+dist.init_process_group("gloo")
+# the paper's arrangement: rank m holds replica m; one all-reduce (sum) of the parameters per round
+w = inputs.WORKLOADS["C1"].scaled(5003)
+x_all = inputs.replicas(w)[:world, :w.d]                 # every rank could draw all, but uses only its own
+mine = np.ascontiguousarray(x_all[rank])
+reduced = torch.from_numpy(mine.copy())
+dist.all_reduce(reduced)                                 # the one collective of the round
+out, r = oracle.worker_update(mine, reduced.numpy(), 1.0 / world, w.alpha, w.lam)
+ref, r_ref = oracle.consensus(np.ascontiguousarray(x_all), w.alpha, w.lam)
+ok = bool(abs(r - r_ref[rank]) <= 1e-6 * r_ref[rank] and np.abs(out.astype(np.float64) - ref[rank]).max() <= 2e-8)
+oks = [None] * world
+dist.all_gather_object(oks, ok)
+if rank == 0:
+    print(json.dumps({"ok": oks}))
+dist.destroy_process_group()
+"""
+
+
+def test_two_ranks_one_replica_each(tmp_path):
+    """Rank m holds replica m, the parameters are all-reduced once, and each rank's own update
+    (the oracle's one-worker form) reproduces its row of the oracle's round on both replicas."""
+    script = tmp_path / "worker_per_rank.py"
+    script.write_text(WORKER_PER_RANK)
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+           "--master-addr", "127.0.0.1", "--master-port", "29535", str(script), ROOT]
+    run = subprocess.run(cmd, capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert run.returncode == 0, run.stderr[-2000:]
+    out = json.loads([l for l in run.stdout.splitlines() if l.startswith("{")][-1])
+    assert out["ok"] == [True, True]

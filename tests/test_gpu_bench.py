@@ -68,3 +68,10 @@ def test_column_shard_line_on_one_gpu(capsys):
     check_common(line, 3)
     assert line["scaling"] == "strong" and "column shards" in line["parallelism"]
     assert line["gpu_launches"] == 3 * 2 * 3                # distance, sum, update per step
+
+
+def test_worker_per_gpu_line_on_one_gpu(capsys):
+    line = run_bench(capsys, ["--workload", "C4", "--d", "2000003", "--shard", "workers"])
+    assert line["roofline"]["algorithmic_bytes_per_launch"] == 5 * 2000003 * 4
+    assert line["scaling"] == "strong" and "one replica" in line["parallelism"]
+    assert line["gpu_launches"] == 3 * 2 and 0 < line["roofline"]["frac"] < 2.0 and len(line["norms_last_round"]) == 1

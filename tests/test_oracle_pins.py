@@ -369,3 +369,35 @@ def test_adamw_matches_library_adamw(oracle):
     xa, aa, ba = oracle.adamw_steps_f64(x0, z, z, grads[:3], lr, b1, b2, eps, wd)
     xb, ab, bb = oracle.adamw_steps_f64(xa, aa, ba, grads[3:], lr, b1, b2, eps, wd, first_step=4)
     assert np.array_equal(xb, x64) and np.array_equal(ab, a64) and np.array_equal(bb, b64)
+
+
+# ---------------------------------------------------------------- one worker given the average
+
+def test_worker_update_hand_cases(oracle):
+    """By hand from the single-line update: x = (0, 0), x_A = (3, 4): r = 5.  alpha = 1/8, lambda = 5/8
+    (both exact in fp32, lambda / alpha = 5) is the fixed point (c = 0); alpha = 0.5, lambda = 0 moves half
+    way; alpha = 0, lambda = 1 moves one
+    unit AWAY from x_A along (x - x_A)/r = (-0.6, -0.8)."""
+    x, red = np.zeros(2, dtype=np.float32), np.array([6.0, 8.0], dtype=np.float32)
+    out, r = oracle.worker_update(x, red, 0.5, 0.125, 0.625)
+    assert r == 5.0 and np.array_equal(out, x)
+    out, r = oracle.worker_update(x, red, 0.5, 0.5, 0.0)
+    assert np.array_equal(out, np.array([1.5, 2.0], dtype=np.float32))
+    out, r = oracle.worker_update(x, red, 0.5, 0.0, 1.0)
+    np.testing.assert_allclose(out, [-0.6, -0.8], rtol=1e-7)
+    out, r = oracle.worker_update(red, red, 1.0, 0.3, 0.7)          # the worker sits on the average
+    assert r == 0.0 and np.array_equal(out, red)
+
+
+def test_worker_update_is_one_row_of_the_round(oracle):
+    """Every worker applying its own update with the shared average reproduces the round on
+    all replicas (the average handed over as fp32, hence a few fp32 ulps of slack)."""
+    rng = np.random.default_rng(11)
+    M, d = 5, 4001
+    x = (rng.standard_normal(d) * 0.02 + rng.standard_normal((M, d)) * 1e-3).astype(np.float32)
+    ref, r_ref = oracle.consensus(x, 0.2, 0.05)
+    total = x.astype(np.float64).sum(axis=0).astype(np.float32)
+    for m in range(M):
+        out, r = oracle.worker_update(x[m], total, 1.0 / M, 0.2, 0.05)
+        assert abs(r - r_ref[m]) <= 1e-6 * r_ref[m]
+        np.testing.assert_allclose(out, ref[m], rtol=0, atol=2e-8)
