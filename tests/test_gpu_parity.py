@@ -399,3 +399,31 @@ def test_runs_on_a_side_stream(oracle):
         binding.dppf_consensus(x, 0.3, 0.02, norms_out=norms, d=d)
     s.synchronize()
     assert_parity(x.cpu().numpy(), norms.cpu().numpy(), ref, r_ref, d)
+
+
+def test_calls_on_two_streams_with_their_own_workspaces_do_not_interfere(oracle):
+    """Two independent replica sets, each with its own workspace, driven from two streams at once
+    (cooperative launches of the two take turns on the GPU): both match the oracle."""
+    import torch
+    _, binding = require_gpu()
+    d = 1_500_003
+    xs_np = [random_replicas(4, d, seed=51), random_replicas(8, d, seed=52)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    xs, norms, wss = [], [], []
+    for x_np in xs_np:
+        xs.append(to_dev(x_np))
+        norms.append(torch.zeros(3, x_np.shape[0], device="cuda"))
+        wss.append(binding.alloc_workspace(x_np.shape[0], d))
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for i, s in enumerate(streams):
+            with torch.cuda.stream(s):
+                binding.dppf_consensus(xs[i], 0.1, 0.01, norms_out=norms[i][rep], ws=wss[i], d=d)
+    for s in streams:
+        s.synchronize()
+    for i, x_np in enumerate(xs_np):
+        ref = x_np
+        for rep in range(3):
+            ref, r_ref = oracle.consensus(ref, 0.1, 0.01, d=d)
+            assert np.all(np.abs(norms[i][rep].cpu().numpy() - r_ref) <= 1e-5 * r_ref)
+        assert_parity(xs[i].cpu().numpy(), norms[i][2].cpu().numpy(), ref, r_ref, d)
