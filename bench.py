@@ -97,6 +97,7 @@ NCU_TRAFFIC = {
     ("C3", 25_557_032, "fused_round_kernel_staged"): 2.746e9,
     ("C4", 86_567_656, "general_round_kernel"): 4.004e9,
     ("C4", 86_567_656, "adamw_round_kernel"): 12.365e9,
+    ("C4", 86_567_656, "worker_round_kernel"): 1.583e9,
 }
 
 
